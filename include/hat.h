@@ -1,0 +1,212 @@
+/*
+ * hat.h -- C ABI of the HAT chunk-attention library (sm_100a).
+ *
+ * The library implements one step of a decoder layer of the cloud-side middle
+ * submodel of HAT: for a ragged batch of requests coming from many end
+ * devices, store the chunk's new keys/values in each request's paged KV cache
+ * and compute causal attention of the chunk's query rows against that cache.
+ * A chunk is either a prompt chunk (prompt chunking, Sec. 2.1 "Batched
+ * Inference" and Sec. 3.3) or the short draft sequence sent up for
+ * verification in a single inference step (Sec. 2.1 "Speculative Decoding",
+ * Sec. 3.4).  Paging of the cache through a block table is what Sec. 4.1 calls
+ * page attention.
+ *
+ * Conventions
+ *   - Every function returns an int status: HAT_OK (0) or a negative error.
+ *     No exception or abort crosses this boundary.
+ *   - "host" / "device" on each pointer says where the memory must live.
+ *   - The caller owns every buffer; the library owns only hat_plan objects.
+ *   - hat_kv_append and hat_chunk_attention allocate nothing, never
+ *     synchronise, and enqueue all work on the given CUDA stream
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - All argument errors are detected on the host before any launch.
+ *   - Layout of packed activations (q, k_new, v_new, out): row-major
+ *     [T][num_heads][head_dim], T = sum of chunk_len; request r owns rows
+ *     cu_chunk[r] .. cu_chunk[r+1]-1.  lse is [T][num_heads].
+ */
+#ifndef HAT_H_
+#define HAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HAT_VERSION 100
+
+/* status codes */
+#define HAT_OK                        0
+#define HAT_ERR_INVALID_ARG          -1  /* null pointer, negative count, cu_chunk inconsistent with chunk_len */
+#define HAT_ERR_UNSUPPORTED          -2  /* dtype, head_dim, page_size, head counts or strides outside what is built */
+#define HAT_ERR_OUT_OF_RANGE         -3  /* page id outside the pool, table too short, page written by two requests */
+#define HAT_ERR_WORKSPACE_TOO_SMALL  -4
+#define HAT_ERR_CUDA                 -5  /* a CUDA runtime call failed; see hat_last_cuda_error */
+#define HAT_ERR_DEVICE_TIMEOUT       -6  /* a bounded device-side wait gave up (reported by hat_last_device_status) */
+#define HAT_ERR_TOO_LARGE            -7  /* a size exceeds a documented fixed maximum */
+
+#define HAT_DTYPE_FP16 0
+#define HAT_DTYPE_BF16 1
+
+/* hat_batch_desc.flags */
+#define HAT_PLAN_HOST_ONLY 1u   /* build and validate the plan but upload nothing (no CUDA call); such a plan
+                                   can be inspected with hat_plan_get_info but not launched */
+
+/*
+ * Geometry of the KV cache (Sec. 2.1: keys and values of all previously
+ * processed tokens; Sec. 4.1: paged).  Logical token p of a request lives in
+ * page block_table[r][p / page_size], slot p % page_size.  Element (page, slot,
+ * head, c) of a pool is at element offset
+ *     page*stride_page + slot*stride_token + head*stride_head + c.
+ * Strides are in elements and must be multiples of 8 (16-byte vectors);
+ * head_dim is contiguous.  Two layouts are typical:
+ *   paged      [page][head][slot][d]: stride_token=d, stride_head=page_size*d, stride_page=heads*page_size*d
+ *   contiguous [token][head][d] with an identity block table:
+ *              stride_token=heads*d, stride_head=d, stride_page=page_size*heads*d
+ */
+typedef struct hat_cache_desc {
+    void*   k_pool;        /* device, 16-byte aligned; may be NULL for hat_plan_create */
+    void*   v_pool;        /* device, 16-byte aligned; may be NULL for hat_plan_create */
+    int32_t dtype;         /* HAT_DTYPE_FP16 | HAT_DTYPE_BF16 (q, k_new, v_new use the same type) */
+    int32_t num_pages;     /* pages in each pool */
+    int32_t page_size;     /* tokens per page; 16 is the only size built */
+    int32_t num_kv_heads;  /* must equal num_q_heads (multi-head attention) */
+    int32_t head_dim;      /* 64 or 128 */
+    int32_t reserved;      /* 0 */
+    int64_t stride_page;
+    int64_t stride_token;
+    int64_t stride_head;
+} hat_cache_desc;
+
+/*
+ * One batch = one inference step over chunks from many devices (Sec. 2.1
+ * continuous batching; Sec. 3.1).  All four arrays are HOST memory and are
+ * copied by hat_plan_create (they may be freed afterwards).
+ *   cu_chunk    [num_requests+1]  exclusive prefix sum of chunk_len, cu_chunk[0]=0
+ *   prefix_len  [num_requests]    tokens already in the request's cache (>=0).  After a round in which
+ *                                 drafts were rejected the caller simply passes the accepted length:
+ *                                 stale slots beyond it are overwritten by the next append (Sec. 3.4)
+ *   chunk_len   [num_requests]    rows of this chunk (>=0; 0 is a valid no-op)
+ *   block_table [num_requests][max_pages] physical page ids; entries at or beyond
+ *                                 ceil((prefix_len+chunk_len)/page_size) are ignored
+ */
+typedef struct hat_batch_desc {
+    int32_t        num_requests;
+    int32_t        num_q_heads;
+    int32_t        max_pages;
+    uint32_t       flags;
+    const int32_t* cu_chunk;
+    const int32_t* prefix_len;
+    const int32_t* chunk_len;
+    const int32_t* block_table;
+} hat_batch_desc;
+
+typedef struct hat_plan hat_plan;
+
+/* What the host-side scheduler decided for a batch (for tests, tuning and reports). */
+typedef struct hat_plan_info {
+    int32_t num_requests;
+    int32_t total_rows;          /* T */
+    int32_t num_verify_requests; /* chunk_len in [1, 16]: split-KV streaming kernel */
+    int32_t num_prefill_requests;/* chunk_len > 16: tile kernel */
+    int32_t num_verify_items;    /* CTAs per head of the streaming kernel */
+    int32_t num_prefill_items;   /* CTAs per head of the tile kernel */
+    int32_t num_merge_rows;      /* rows whose result is merged from several key ranges */
+    int32_t max_splits;          /* largest number of key ranges any request was cut into */
+    int32_t verify_split_len;    /* tokens per key range, streaming kernel */
+    int32_t prefill_split_len;   /* tokens per key range, tile kernel (0 = unsplit) */
+    int32_t prefill_tile_rows;   /* query rows per CTA of the tile kernel */
+    int32_t prefill_kernel;      /* 0 = mma.sync tile kernel, 1 = tcgen05 tile kernel */
+    int64_t workspace_bytes;
+    int64_t attn_flops;          /* 4*d*H*sum_r [C_r*P_r + C_r*(C_r+1)/2] */
+    int64_t kv_read_bytes;       /* 2*sum_r (P_r+C_r)*H*d*elem: every visible K and V row read once per head */
+} hat_plan_info;
+
+const char* hat_status_string(int status);
+int         hat_version(void);
+
+/* cudaError_t of the most recent failing CUDA call made by this library on the calling thread (0 if none). */
+int         hat_last_cuda_error(void);
+
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t     hat_launch_count(void);
+
+/*
+ * Validate a batch and schedule it (Sec. 2.1 "Batched Inference": the batch
+ * mixes prefill chunks and decode-phase requests; cost follows the batched
+ * token size).  Requests with chunk_len <= 16 take the split-KV streaming
+ * path, longer chunks the tile path; long key ranges are cut so that every SM
+ * has work, and rows cut into several ranges are merged afterwards.
+ * Unless HAT_PLAN_HOST_ONLY is set the schedule is uploaded to the current
+ * device (one cudaMalloc + one synchronous copy).  A plan can be reused for
+ * every layer of the step and must be destroyed with hat_plan_destroy.
+ * Errors: INVALID_ARG, UNSUPPORTED, OUT_OF_RANGE, CUDA.  *out is NULL on error.
+ */
+int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, hat_plan** out);
+int hat_plan_get_info(const hat_plan* plan, hat_plan_info* out);
+int hat_plan_workspace_bytes(const hat_plan* plan, size_t* out);
+int hat_plan_destroy(hat_plan* plan);   /* NULL is accepted */
+
+/*
+ * KV append (Sec. 2.1, KV cache).  For request r, chunk row i and head h the
+ * 16-bit patterns k_new[cu_chunk[r]+i][h][:] and v_new[...] are stored,
+ * bit-exactly, at logical token prefix_len[r]+i of the request's cache.  No
+ * other slot of the pools is written.
+ *   cache          geometry + device pools (both non-NULL)
+ *   k_new, v_new   device, [T][heads][head_dim], 16-byte aligned
+ */
+int hat_kv_append(const hat_cache_desc* cache, const hat_plan* plan,
+                  const void* k_new, const void* v_new, void* stream);
+
+/*
+ * Chunk attention (Sec. 2.1 self-attention over the KV cache; Sec. 2.1 / 3.3
+ * prompt chunks; Sec. 3.4 draft verification).  For packed row t = cu_chunk[r]+i
+ * and head h, with g = prefix_len[r]+i and keys/values j = 0..g read through
+ * the block table:
+ *     s_j = sm_scale * <q[t][h], K_j[h]>
+ *     out[t][h][:] = sum_j softmax(s)_j * V_j[h][:]        (fp32)
+ *     lse[t][h]    = ln sum_j exp(s_j)                     (fp32, natural log)
+ * The chunk's own K/V must be in the cache: either call hat_kv_append first, or
+ * pass k_new/v_new here (both non-NULL), which performs the same append on
+ * `stream` before attending.
+ *   q                device [T][heads][head_dim], same dtype as the cache, 16-byte aligned
+ *   out, lse         device fp32, 16-byte aligned
+ *   sm_scale         <= 0 or NaN selects 1/sqrt(head_dim)
+ *   workspace        device, 256-byte aligned, at least hat_plan_workspace_bytes; may be NULL if that is 0.
+ *                    Concurrent calls must use different workspaces.
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, CUDA.
+ */
+int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q,
+                        const void* k_new, const void* v_new,
+                        float* out, float* lse, float sm_scale,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same step for a caller whose activations live in HOST memory (pinned
+ * memory makes the copies asynchronous).  Copies q, k_new, v_new to `staging`,
+ * appends, attends, copies out and lse back, all on `stream`, and returns
+ * without synchronising: the host results are valid once the stream is.
+ *   q_host, k_new_host, v_new_host   host [T][heads][head_dim] 16-bit
+ *   out_host [T][heads][head_dim], lse_host [T][heads]   host fp32
+ *   staging        device, 256-byte aligned, >= hat_plan_staging_bytes
+ *   workspace      as for hat_chunk_attention
+ */
+int hat_plan_staging_bytes(const hat_plan* plan, size_t* out);
+int hat_chunk_attention_host(const hat_cache_desc* cache, const hat_plan* plan,
+                             const void* q_host, const void* k_new_host, const void* v_new_host,
+                             float* out_host, float* lse_host, float sm_scale,
+                             void* staging, size_t staging_bytes,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Read the device-side status word of a plan (synchronises `stream`).  *out is
+ * HAT_OK, or HAT_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up
+ * since the plan was created; results of such a call are undefined.
+ */
+int hat_last_device_status(const hat_plan* plan, void* stream, int* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HAT_H_ */

@@ -1,0 +1,475 @@
+// C ABI of the library: status strings, host-side validation and scheduling (the plan), and the
+// entry points that enqueue the kernels.  Declarations and argument contracts are in include/hat.h.
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "hat_internal.h"
+
+namespace hat {
+
+static thread_local int g_last_cuda_error = 0;
+static std::atomic<int64_t> g_launches{0};
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return HAT_ERR_CUDA;
+}
+
+static int env_int(const char* name, int dflt) {
+    const char* s = std::getenv(name);
+    if (!s || !*s) return dflt;
+    char* end = nullptr;
+    long v = std::strtol(s, &end, 10);
+    return (end && *end == 0) ? (int)v : dflt;
+}
+
+static inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+static inline int ceil_div(int x, int m) { return (x + m - 1) / m; }
+
+static int check_cache_geometry(const hat_cache_desc* c) {
+    if (!c) return HAT_ERR_INVALID_ARG;
+    if (c->num_pages < 0) return HAT_ERR_INVALID_ARG;
+    if (c->dtype != HAT_DTYPE_FP16 && c->dtype != HAT_DTYPE_BF16) return HAT_ERR_UNSUPPORTED;
+    if (c->page_size != kPageSize) return HAT_ERR_UNSUPPORTED;
+    if (c->head_dim != 64 && c->head_dim != 128) return HAT_ERR_UNSUPPORTED;
+    if (c->num_kv_heads <= 0) return HAT_ERR_INVALID_ARG;
+    if (c->stride_page <= 0 || c->stride_token <= 0 || c->stride_head <= 0) return HAT_ERR_INVALID_ARG;
+    if (c->stride_page % 8 || c->stride_token % 8 || c->stride_head % 8) return HAT_ERR_UNSUPPORTED;
+    return HAT_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Cut the key range [0, kv_end) of one tile into pieces of `split_len` keys (the last piece takes the
+// remainder) and emit one work item per piece.
+static void emit_tile(hat_plan* p, std::vector<WorkItem>& items, int req, int row0, int rows_valid,
+                      int kv_end, int split_len) {
+    int nsplit = (split_len > 0) ? ceil_div(kv_end, split_len) : 1;
+    if (nsplit <= 1) {
+        items.push_back(WorkItem{req, row0, 0, kv_end, -1, 0, 0, 0});
+        return;
+    }
+    int64_t base = p->part_rows;
+    for (int s = 0; s < nsplit; ++s) {
+        int b = s * split_len, e = std::min(kv_end, b + split_len);
+        items.push_back(WorkItem{req, row0, b, e, (int32_t)(base + (int64_t)s * rows_valid), 0, 0, 0});
+    }
+    int row_base = p->cu_chunk[req] + row0;
+    for (int i = 0; i < rows_valid; ++i)
+        p->merge_rows.push_back(MergeRow{row_base + i, (int32_t)(base + i), rows_valid, nsplit});
+    p->part_rows += (int64_t)nsplit * rows_valid;
+    p->info.max_splits = std::max(p->info.max_splits, nsplit);
+}
+
+static int split_len_for(int kv_end, int wanted, int granule) {
+    // at most kMaxSplits pieces per tile
+    int least = round_up(ceil_div(kv_end, kMaxSplits), granule);
+    return std::max(wanted, least);
+}
+
+static void schedule(hat_plan* p, int num_sms) {
+    const int H = p->num_heads;
+    const int R = p->num_requests;
+    hat_plan_info& info = p->info;
+
+    const int verify_max_rows = 16;
+    const int tile_rows = 64;                     // mma.sync tile kernel: 4 warps x 16 rows
+    info.prefill_tile_rows = tile_rows;
+    info.prefill_kernel = 0;
+
+    // ---- streaming (verify-class) requests: fixed-length key ranges, shortened until the SMs are covered
+    int64_t verify_tokens = 0;
+    for (int r = 0; r < R; ++r) {
+        int C = p->chunk_len[r];
+        if (C >= 1 && C <= verify_max_rows) {
+            verify_tokens += p->prefix_len[r] + C;
+            info.num_verify_requests++;
+        } else if (C > verify_max_rows) {
+            info.num_prefill_requests++;
+        }
+    }
+    int vsplit = env_int("HAT_VERIFY_SPLIT_LEN", 0);
+    if (vsplit <= 0) {
+        vsplit = 512;
+        const int64_t want_ctas = (int64_t)num_sms * 8;
+        while (vsplit > 64 && (verify_tokens / vsplit + info.num_verify_requests) * H < want_ctas) vsplit /= 2;
+    }
+    vsplit = std::max(kPageSize, round_up(vsplit, kPageSize));
+    info.verify_split_len = vsplit;
+
+    // ---- tile (prefill-class) requests: cut keys only when there are too few tiles to cover the SMs
+    int64_t tiles = 0, tile_keys = 0;
+    for (int r = 0; r < R; ++r) {
+        int C = p->chunk_len[r];
+        if (C <= verify_max_rows) continue;
+        for (int row0 = 0; row0 < C; row0 += tile_rows) {
+            tiles++;
+            tile_keys += p->prefix_len[r] + std::min(C, row0 + tile_rows);
+        }
+    }
+    int psplit = env_int("HAT_PREFILL_SPLIT_LEN", -1);
+    if (psplit < 0) {
+        psplit = 0;
+        const int64_t want_ctas = (int64_t)num_sms * 2;
+        if (tiles > 0 && tiles * H < want_ctas) {
+            // aim for want_ctas pieces of equal length, not shorter than 256 keys
+            int64_t pieces = ceil_div((int)want_ctas, H);
+            psplit = std::max<int64_t>(256, round_up((int)ceil_div((int)tile_keys, (int)pieces), 64));
+        }
+    }
+    if (psplit > 0) psplit = round_up(psplit, 64);
+    info.prefill_split_len = psplit;
+
+    for (int r = 0; r < R; ++r) {
+        int C = p->chunk_len[r], P = p->prefix_len[r];
+        if (C <= 0) continue;
+        if (C <= verify_max_rows) {
+            int kv_end = P + C;
+            emit_tile(p, p->verify_items, r, 0, C, kv_end, split_len_for(kv_end, vsplit, kPageSize));
+        } else {
+            for (int row0 = 0; row0 < C; row0 += tile_rows) {
+                int rows_valid = std::min(tile_rows, C - row0);
+                int kv_end = P + row0 + rows_valid;
+                int sl = psplit > 0 ? split_len_for(kv_end, psplit, 64) : 0;
+                emit_tile(p, p->prefill_items, r, row0, rows_valid, kv_end, sl);
+            }
+        }
+    }
+    // longest pieces first so the tail of the grid is made of short ones
+    auto longer = [](const WorkItem& a, const WorkItem& b) {
+        return (a.kv_end - a.kv_begin) > (b.kv_end - b.kv_begin);
+    };
+    std::stable_sort(p->verify_items.begin(), p->verify_items.end(), longer);
+    std::stable_sort(p->prefill_items.begin(), p->prefill_items.end(), longer);
+
+    info.num_verify_items = (int32_t)p->verify_items.size();
+    info.num_prefill_items = (int32_t)p->prefill_items.size();
+    info.num_merge_rows = (int32_t)p->merge_rows.size();
+    const int64_t d = p->head_dim;
+    int64_t part_out_bytes = round_up((int)0, 1) + p->part_rows * H * d * 4;
+    part_out_bytes = (part_out_bytes + 255) / 256 * 256;
+    info.workspace_bytes = p->part_rows ? part_out_bytes + ((p->part_rows * H * 4 + 255) / 256 * 256) : 0;
+}
+
+template <typename T>
+static size_t blob_append(std::vector<char>& blob, const std::vector<T>& v) {
+    size_t off = (blob.size() + 255) / 256 * 256;
+    blob.resize(off + std::max<size_t>(v.size() * sizeof(T), 16));
+    if (!v.empty()) std::memcpy(blob.data() + off, v.data(), v.size() * sizeof(T));
+    return off;
+}
+
+static int upload(hat_plan* p) {
+    std::vector<char> blob;
+    size_t o_cu = blob_append(blob, p->cu_chunk);
+    size_t o_pl = blob_append(blob, p->prefix_len);
+    size_t o_cl = blob_append(blob, p->chunk_len);
+    size_t o_bt = blob_append(blob, p->block_table);
+    size_t o_rr = blob_append(blob, p->row_req);
+    size_t o_vi = blob_append(blob, p->verify_items);
+    size_t o_pi = blob_append(blob, p->prefill_items);
+    size_t o_mr = blob_append(blob, p->merge_rows);
+    std::vector<int32_t> status(4, 0);
+    size_t o_st = blob_append(blob, status);
+
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaMalloc(&p->dev_blob, blob.size());
+    if (e != cudaSuccess) { p->dev_blob = nullptr; return cuda_fail(e); }
+    e = cudaMemcpy(p->dev_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail(e);
+    char* base = static_cast<char*>(p->dev_blob);
+    DevicePlan& d = p->dev;
+    d.cu_chunk = reinterpret_cast<const int32_t*>(base + o_cu);
+    d.prefix_len = reinterpret_cast<const int32_t*>(base + o_pl);
+    d.chunk_len = reinterpret_cast<const int32_t*>(base + o_cl);
+    d.block_table = reinterpret_cast<const int32_t*>(base + o_bt);
+    d.row_req = reinterpret_cast<const int32_t*>(base + o_rr);
+    d.verify_items = reinterpret_cast<const WorkItem*>(base + o_vi);
+    d.prefill_items = reinterpret_cast<const WorkItem*>(base + o_pi);
+    d.merge_rows = reinterpret_cast<const MergeRow*>(base + o_mr);
+    d.status = reinterpret_cast<int32_t*>(base + o_st);
+    d.max_pages = p->max_pages;
+    d.num_heads = p->num_heads;
+    d.total_rows = p->total_rows;
+    return HAT_OK;
+}
+
+static int check_call(const hat_cache_desc* cache, const hat_plan* plan) {
+    if (!cache || !plan) return HAT_ERR_INVALID_ARG;
+    if (plan->host_only) return HAT_ERR_INVALID_ARG;
+    int st = check_cache_geometry(cache);
+    if (st != HAT_OK) return st;
+    if (cache->dtype != plan->dtype || cache->num_pages != plan->num_pages ||
+        cache->num_kv_heads != plan->num_heads || cache->head_dim != plan->head_dim)
+        return HAT_ERR_INVALID_ARG;
+    if (!cache->k_pool || !cache->v_pool) return HAT_ERR_INVALID_ARG;
+    if (!aligned(cache->k_pool, 16) || !aligned(cache->v_pool, 16)) return HAT_ERR_INVALID_ARG;
+    return HAT_OK;
+}
+
+static CacheView view_of(const hat_cache_desc* c) {
+    return CacheView{c->k_pool, c->v_pool, c->stride_page, c->stride_token, c->stride_head};
+}
+
+}  // namespace hat
+
+using namespace hat;
+
+extern "C" {
+
+const char* hat_status_string(int status) {
+    switch (status) {
+        case HAT_OK: return "ok";
+        case HAT_ERR_INVALID_ARG: return "invalid argument";
+        case HAT_ERR_UNSUPPORTED: return "unsupported configuration";
+        case HAT_ERR_OUT_OF_RANGE: return "index out of range";
+        case HAT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case HAT_ERR_CUDA: return "CUDA error";
+        case HAT_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case HAT_ERR_TOO_LARGE: return "size exceeds a fixed maximum";
+        default: return "unknown status";
+    }
+}
+
+int hat_version(void) { return HAT_VERSION; }
+int hat_last_cuda_error(void) { return g_last_cuda_error; }
+int64_t hat_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, hat_plan** out) {
+    if (!out) return HAT_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cache || !batch) return HAT_ERR_INVALID_ARG;
+    int st = check_cache_geometry(cache);
+    if (st != HAT_OK) return st;
+    const int R = batch->num_requests;
+    if (R < 0 || batch->max_pages < 0 || batch->num_q_heads <= 0) return HAT_ERR_INVALID_ARG;
+    if (batch->num_q_heads != cache->num_kv_heads) return HAT_ERR_UNSUPPORTED;
+    if (!batch->cu_chunk) return HAT_ERR_INVALID_ARG;
+    if (R > 0 && (!batch->prefix_len || !batch->chunk_len)) return HAT_ERR_INVALID_ARG;
+    if (batch->cu_chunk[0] != 0) return HAT_ERR_INVALID_ARG;
+
+    // shapes
+    int64_t total = 0;
+    for (int r = 0; r < R; ++r) {
+        if (batch->prefix_len[r] < 0 || batch->chunk_len[r] < 0) return HAT_ERR_INVALID_ARG;
+        total += batch->chunk_len[r];
+        if (batch->cu_chunk[r + 1] != total) return HAT_ERR_INVALID_ARG;
+        if ((int64_t)batch->prefix_len[r] + batch->chunk_len[r] > (int64_t)INT32_MAX / 2) return HAT_ERR_TOO_LARGE;
+    }
+    if (total > INT32_MAX / 2) return HAT_ERR_TOO_LARGE;
+
+    // block tables: long enough, inside the pool, and no page written by two requests
+    std::vector<uint8_t> written(cache->num_pages > 0 ? cache->num_pages : 0, 0);
+    for (int r = 0; r < R; ++r) {
+        const int C = batch->chunk_len[r];
+        if (C == 0) continue;
+        const int N = batch->prefix_len[r] + C;
+        const int need = (N + kPageSize - 1) / kPageSize;
+        if (need > batch->max_pages) return HAT_ERR_OUT_OF_RANGE;
+        if (!batch->block_table) return HAT_ERR_INVALID_ARG;
+        const int32_t* row = batch->block_table + (int64_t)r * batch->max_pages;
+        for (int j = 0; j < need; ++j)
+            if (row[j] < 0 || row[j] >= cache->num_pages) return HAT_ERR_OUT_OF_RANGE;
+        for (int j = batch->prefix_len[r] / kPageSize; j < need; ++j) {
+            if (written[row[j]]) return HAT_ERR_OUT_OF_RANGE;
+            written[row[j]] = 1;
+        }
+    }
+
+    hat_plan* p = new (std::nothrow) hat_plan();
+    if (!p) return HAT_ERR_INVALID_ARG;
+    p->dtype = cache->dtype;
+    p->num_pages = cache->num_pages;
+    p->num_heads = cache->num_kv_heads;
+    p->head_dim = cache->head_dim;
+    p->max_pages = batch->max_pages;
+    p->num_requests = R;
+    p->total_rows = (int32_t)total;
+    p->host_only = (batch->flags & HAT_PLAN_HOST_ONLY) != 0;
+    p->device = -1;
+    p->part_rows = 0;
+    p->dev_blob = nullptr;
+    std::memset(&p->info, 0, sizeof p->info);
+    std::memset(&p->dev, 0, sizeof p->dev);
+    p->cu_chunk.assign(batch->cu_chunk, batch->cu_chunk + R + 1);
+    p->prefix_len.assign(batch->prefix_len, batch->prefix_len + R);
+    p->chunk_len.assign(batch->chunk_len, batch->chunk_len + R);
+    if (batch->block_table && batch->max_pages > 0)
+        p->block_table.assign(batch->block_table, batch->block_table + (int64_t)R * batch->max_pages);
+    p->row_req.resize(total);
+    for (int r = 0; r < R; ++r)
+        for (int t = p->cu_chunk[r]; t < p->cu_chunk[r + 1]; ++t) p->row_req[t] = r;
+
+    p->info.num_requests = R;
+    p->info.total_rows = (int32_t)total;
+    const int64_t d = p->head_dim, H = p->num_heads;
+    for (int r = 0; r < R; ++r) {
+        const int64_t C = p->chunk_len[r], P = p->prefix_len[r];
+        if (C == 0) continue;
+        p->info.attn_flops += 4 * d * H * (C * P + C * (C + 1) / 2);
+        p->info.kv_read_bytes += 2 * (P + C) * H * d * 2;
+    }
+
+    int num_sms = 148;
+    if (!p->host_only) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+    }
+    schedule(p, num_sms);
+
+    if (!p->host_only) {
+        st = upload(p);
+        if (st != HAT_OK) { hat_plan_destroy(p); return st; }
+    }
+    *out = p;
+    return HAT_OK;
+}
+
+int hat_plan_get_info(const hat_plan* plan, hat_plan_info* out) {
+    if (!plan || !out) return HAT_ERR_INVALID_ARG;
+    *out = plan->info;
+    return HAT_OK;
+}
+
+int hat_plan_workspace_bytes(const hat_plan* plan, size_t* out) {
+    if (!plan || !out) return HAT_ERR_INVALID_ARG;
+    *out = (size_t)plan->info.workspace_bytes;
+    return HAT_OK;
+}
+
+int hat_plan_destroy(hat_plan* plan) {
+    if (!plan) return HAT_OK;
+    int st = HAT_OK;
+    if (plan->dev_blob) {
+        cudaError_t e = cudaFree(plan->dev_blob);
+        if (e != cudaSuccess) st = cuda_fail(e);
+    }
+    delete plan;
+    return st;
+}
+
+int hat_kv_append(const hat_cache_desc* cache, const hat_plan* plan, const void* k_new, const void* v_new,
+                  void* stream) {
+    int st = check_call(cache, plan);
+    if (st != HAT_OK) return st;
+    if (plan->total_rows == 0) return HAT_OK;
+    if (!k_new || !v_new || !aligned(k_new, 16) || !aligned(v_new, 16)) return HAT_ERR_INVALID_ARG;
+    cudaError_t e = launch_kv_append(plan, view_of(cache), cache->k_pool, cache->v_pool, k_new, v_new,
+                                     static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? HAT_OK : cuda_fail(e);
+}
+
+int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
+                        const void* v_new, float* out, float* lse, float sm_scale, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    int st = check_call(cache, plan);
+    if (st != HAT_OK) return st;
+    if ((k_new == nullptr) != (v_new == nullptr)) return HAT_ERR_INVALID_ARG;
+    if (plan->total_rows == 0) return HAT_OK;
+    if (!q || !out || !lse) return HAT_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(lse, 16)) return HAT_ERR_INVALID_ARG;
+    if (k_new && (!aligned(k_new, 16) || !aligned(v_new, 16))) return HAT_ERR_INVALID_ARG;
+    const size_t need = (size_t)plan->info.workspace_bytes;
+    if (need > 0) {
+        if (!workspace || !aligned(workspace, 256)) return HAT_ERR_INVALID_ARG;
+        if (workspace_bytes < need) return HAT_ERR_WORKSPACE_TOO_SMALL;
+    }
+    if (!(sm_scale > 0.f) || !std::isfinite(sm_scale)) sm_scale = 1.0f / std::sqrt((float)plan->head_dim);
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (k_new) {
+        e = launch_kv_append(plan, view_of(cache), cache->k_pool, cache->v_pool, k_new, v_new, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    AttnArgs a;
+    a.plan = plan->dev;
+    a.cache = view_of(cache);
+    a.q = q;
+    a.out = out;
+    a.lse = lse;
+    a.part_out = static_cast<float*>(workspace);
+    const int64_t H = plan->num_heads, d = plan->head_dim;
+    const size_t part_out_bytes = ((size_t)plan->part_rows * H * d * 4 + 255) / 256 * 256;
+    a.part_lse = need ? reinterpret_cast<float*>(static_cast<char*>(workspace) + part_out_bytes) : nullptr;
+    a.scale_log2 = sm_scale * 1.4426950408889634f;
+
+    if (!plan->prefill_items.empty()) {
+        e = launch_attn_mma(plan, a, /*verify_class=*/false, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (!plan->verify_items.empty()) {
+        e = launch_attn_mma(plan, a, /*verify_class=*/true, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (!plan->merge_rows.empty()) {
+        e = launch_merge(plan, a, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return HAT_OK;
+}
+
+int hat_plan_staging_bytes(const hat_plan* plan, size_t* out) {
+    if (!plan || !out) return HAT_ERR_INVALID_ARG;
+    const size_t T = plan->total_rows, H = plan->num_heads, d = plan->head_dim;
+    const size_t act16 = (T * H * d * 2 + 255) / 256 * 256;
+    const size_t out32 = (T * H * d * 4 + 255) / 256 * 256;
+    const size_t lse32 = (T * H * 4 + 255) / 256 * 256;
+    *out = 3 * act16 + out32 + lse32;
+    return HAT_OK;
+}
+
+int hat_chunk_attention_host(const hat_cache_desc* cache, const hat_plan* plan, const void* q_host,
+                             const void* k_new_host, const void* v_new_host, float* out_host, float* lse_host,
+                             float sm_scale, void* staging, size_t staging_bytes, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    int st = check_call(cache, plan);
+    if (st != HAT_OK) return st;
+    if (plan->total_rows == 0) return HAT_OK;
+    if (!q_host || !k_new_host || !v_new_host || !out_host || !lse_host) return HAT_ERR_INVALID_ARG;
+    size_t need = 0;
+    hat_plan_staging_bytes(plan, &need);
+    if (!staging || !aligned(staging, 256)) return HAT_ERR_INVALID_ARG;
+    if (staging_bytes < need) return HAT_ERR_WORKSPACE_TOO_SMALL;
+    const size_t T = plan->total_rows, H = plan->num_heads, d = plan->head_dim;
+    const size_t act_bytes = T * H * d * 2, out_bytes = T * H * d * 4, lse_bytes = T * H * 4;
+    const size_t act16 = (act_bytes + 255) / 256 * 256, out32 = (out_bytes + 255) / 256 * 256;
+    char* base = static_cast<char*>(staging);
+    void* dq = base;
+    void* dk = base + act16;
+    void* dv = base + 2 * act16;
+    float* dout = reinterpret_cast<float*>(base + 3 * act16);
+    float* dlse = reinterpret_cast<float*>(base + 3 * act16 + out32);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(dq, q_host, act_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(dk, k_new_host, act_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(dv, v_new_host, act_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    st = hat_chunk_attention(cache, plan, dq, dk, dv, dout, dlse, sm_scale, workspace, workspace_bytes, stream);
+    if (st != HAT_OK) return st;
+    if ((e = cudaMemcpyAsync(out_host, dout, out_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(lse_host, dlse, lse_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    return HAT_OK;
+}
+
+int hat_last_device_status(const hat_plan* plan, void* stream, int* out) {
+    if (!plan || !out || plan->host_only) return HAT_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, plan->dev.status, sizeof word, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *out = word == 0 ? HAT_OK : HAT_ERR_DEVICE_TIMEOUT;
+    return HAT_OK;
+}
+
+}  // extern "C"

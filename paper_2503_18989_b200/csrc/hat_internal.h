@@ -1,0 +1,90 @@
+// Internal declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <vector>
+
+#include "../../include/hat.h"
+
+namespace hat {
+
+constexpr int kPageSize = 16;
+constexpr int kMaxSplits = 32;     // a merged row combines at most this many key ranges (one lane each)
+
+// One CTA's worth of attention work for one head: rows [row0, row0+tile_rows) of request `req`
+// against keys [kv_begin, kv_end).  `part` < 0: the CTA writes the final out/lse rows; otherwise it
+// writes partial results at partial-row index part + (row - 0) for later merging.
+struct WorkItem {
+    int32_t req;
+    int32_t row0;
+    int32_t kv_begin;
+    int32_t kv_end;
+    int32_t part;
+    int32_t pad0, pad1, pad2;
+};
+
+// Rows whose result is merged from `nsplit` partial rows part0 + s*stride, s = 0..nsplit-1.
+struct MergeRow {
+    int32_t row;      // packed row index t
+    int32_t part0;    // partial-row index of split 0
+    int32_t stride;   // partial-row distance between consecutive splits
+    int32_t nsplit;
+};
+
+// Device-resident view of a plan (all pointers device).
+struct DevicePlan {
+    const int32_t*  cu_chunk;
+    const int32_t*  prefix_len;
+    const int32_t*  chunk_len;
+    const int32_t*  block_table;
+    const int32_t*  row_req;        // [T] request of each packed row
+    const WorkItem* verify_items;
+    const WorkItem* prefill_items;
+    const MergeRow* merge_rows;
+    int32_t*        status;         // device status word (0 = ok)
+    int32_t         max_pages;
+    int32_t         num_heads;
+    int32_t         total_rows;
+};
+
+struct CacheView {
+    const void* k_pool;
+    const void* v_pool;
+    int64_t stride_page, stride_token, stride_head;
+};
+
+struct AttnArgs {
+    DevicePlan  plan;
+    CacheView   cache;
+    const void* q;
+    float*      out;          // [T][H][d]
+    float*      lse;          // [T][H]
+    float*      part_out;     // [part_rows][H][d]
+    float*      part_lse;     // [part_rows][H]
+    float       scale_log2;   // sm_scale * log2(e)
+};
+
+}  // namespace hat
+
+struct hat_plan {
+    // geometry the plan was made for
+    int32_t dtype, num_pages, num_heads, head_dim, max_pages, num_requests, total_rows;
+    bool host_only;
+    int device;
+    std::vector<int32_t> cu_chunk, prefix_len, chunk_len, block_table, row_req;
+    std::vector<hat::WorkItem> verify_items, prefill_items;
+    std::vector<hat::MergeRow> merge_rows;
+    int64_t part_rows;          // partial rows in the workspace
+    hat_plan_info info;
+    void* dev_blob;             // one allocation holding every device array
+    hat::DevicePlan dev;
+};
+
+namespace hat {
+// kernel launchers (each returns a cudaError_t from the launch)
+cudaError_t launch_kv_append(const hat_plan* plan, const CacheView& cache, void* k_pool, void* v_pool,
+                             const void* k_new, const void* v_new, cudaStream_t stream);
+cudaError_t launch_attn_mma(const hat_plan* plan, const AttnArgs& args, bool verify_class, cudaStream_t stream);
+cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+void count_launch(int n = 1);
+}  // namespace hat

@@ -1,0 +1,85 @@
+"""Device-side driver for a workload scenario: owns the torch buffers and calls the C-ABI library.
+
+PyTorch is used here for device memory and streams only; every step of the path
+(plan, append, attention, merge) runs inside libhat.so through `binding`.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .workloads import CacheSpec, Scenario, Step
+
+
+def _dev_u16(a: np.ndarray, device) -> torch.Tensor:
+    """uint16 bit patterns -> device tensor (stored as int16; only the bits matter)."""
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(device, non_blocking=False)
+
+
+class DeviceCache:
+    """K and V pools of one layer on the device."""
+
+    def __init__(self, spec: CacheSpec, k_pool: np.ndarray, v_pool: np.ndarray, device="cuda:0"):
+        self.spec = spec
+        self.device = torch.device(device)
+        self.k = _dev_u16(k_pool, self.device)
+        self.v = _dev_u16(v_pool, self.device)
+        self.desc = B.make_cache_desc(spec.dtype, spec.num_pages, spec.num_heads, spec.head_dim,
+                                      spec.stride_page, spec.stride_token, spec.stride_head, self.k, self.v,
+                                      spec.page_size)
+
+    def pools_to_host(self):
+        return (self.k.cpu().numpy().view(np.uint16), self.v.cpu().numpy().view(np.uint16))
+
+
+class DeviceStep:
+    """One batch resident on the device, with its plan, outputs and workspace."""
+
+    def __init__(self, cache: DeviceCache, step: Step):
+        dev = cache.device
+        spec = cache.spec
+        self.cache = cache
+        self.step = step
+        self.plan = B.hat_plan_create(cache.desc, spec.num_heads, step.cu_chunk, step.prefix_len, step.chunk_len,
+                                      step.block_table)
+        self.info = B.hat_plan_get_info(self.plan).as_dict()
+        T, H, d = step.total_rows, spec.num_heads, spec.head_dim
+        self.q = _dev_u16(step.q, dev)
+        self.k_new = _dev_u16(step.k_new, dev)
+        self.v_new = _dev_u16(step.v_new, dev)
+        self.out = torch.full((T, H, d), float("nan"), dtype=torch.float32, device=dev)
+        self.lse = torch.full((T, H), float("nan"), dtype=torch.float32, device=dev)
+        self.workspace_bytes = B.hat_plan_workspace_bytes(self.plan)
+        self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=dev)
+
+    def append(self, stream: int = 0) -> None:
+        B.hat_kv_append(self.cache.desc, self.plan, self.k_new, self.v_new, stream)
+
+    def attend(self, fused_append: bool = True, sm_scale: float = 0.0, stream: int = 0) -> None:
+        B.hat_chunk_attention(self.cache.desc, self.plan, self.q,
+                              self.k_new if fused_append else None, self.v_new if fused_append else None,
+                              self.out, self.lse, sm_scale, self.workspace, self.workspace_bytes, stream)
+
+    def results(self):
+        torch.cuda.synchronize(self.cache.device)
+        return self.out.cpu().numpy(), self.lse.cpu().numpy()
+
+    def close(self):
+        self.plan.close()
+
+
+def run_scenario(sc: Scenario, device="cuda:0", fused_append: bool = True):
+    """Run every step of a scenario in order; returns (cache, [(out, lse) per step])."""
+    cache = DeviceCache(sc.cache, sc.k_pool, sc.v_pool, device)
+    res = []
+    for st in sc.steps:
+        ds = DeviceStep(cache, st)
+        if not fused_append:
+            ds.append()
+        ds.attend(fused_append=fused_append)
+        res.append(ds.results())
+        if B.hat_last_device_status(ds.plan) != B.HAT_OK:
+            raise RuntimeError("device-side wait timed out")
+        ds.close()
+    return cache, res

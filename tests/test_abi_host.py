@@ -1,0 +1,164 @@
+"""Host-side tests of the C-ABI library: it loads, exports what include/hat.h declares, rejects bad
+arguments before any launch, and schedules batches sensibly.  No test here needs a GPU."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2503_18989_b200 import binding as B
+from paper_2503_18989_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "hat.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hat_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(hat_lib):
+    declared = _declared_symbols()
+    assert "hat_kv_append" in declared and "hat_chunk_attention" in declared
+    for name in declared:
+        assert hasattr(hat_lib, name), f"{name} is declared in hat.h but not exported"
+    assert sorted(B.EXPORTS) == declared, "binding and header disagree on the entry points"
+
+
+def test_version_and_status_strings(hat_lib):
+    assert B.hat_version() == 100
+    seen = {B.hat_status_string(s) for s in range(0, -8, -1)}
+    assert len(seen) == 8 and "unknown status" not in seen
+    assert B.hat_status_string(-99) == "unknown status"
+
+
+def _cache(dtype="fp16", num_pages=64, H=4, d=128, **over):
+    spec = W.CacheSpec(dtype, H, d, num_pages, "paged")
+    kw = dict(dtype=dtype, num_pages=num_pages, num_kv_heads=H, head_dim=d, stride_page=spec.stride_page,
+              stride_token=spec.stride_token, stride_head=spec.stride_head)
+    kw.update(over)
+    return B.make_cache_desc(**kw)
+
+
+def _plan(cache, prefix, chunk, table, H=4, cu=None, flags=B.HAT_PLAN_HOST_ONLY):
+    prefix = np.asarray(prefix, np.int32)
+    chunk = np.asarray(chunk, np.int32)
+    if cu is None:
+        cu = np.concatenate([[0], np.cumsum(chunk)]).astype(np.int32)
+    return B.hat_plan_create(cache, H, cu, prefix, chunk, np.asarray(table, np.int32), flags)
+
+
+def _status(fn, *a, **k):
+    try:
+        fn(*a, **k)
+    except B.HatError as e:
+        return e.status
+    return B.HAT_OK
+
+
+def test_plan_rejects_bad_arguments(hat_lib):
+    c = _cache()
+    ok_table = [[0, 1, 2, 3]]
+    assert _status(_plan, c, [10], [20], ok_table) == B.HAT_OK
+    # cu_chunk not the prefix sum of chunk_len
+    assert _status(_plan, c, [10], [20], ok_table, cu=np.array([0, 19], np.int32)) == B.HAT_ERR_INVALID_ARG
+    assert _status(_plan, c, [10], [20], ok_table, cu=np.array([1, 21], np.int32)) == B.HAT_ERR_INVALID_ARG
+    assert _status(_plan, c, [-1], [20], ok_table) == B.HAT_ERR_INVALID_ARG
+    assert _status(_plan, c, [10], [-2], ok_table, cu=np.array([0, -2], np.int32)) == B.HAT_ERR_INVALID_ARG
+    # table too short / page outside the pool / unused entries may be anything
+    assert _status(_plan, c, [60], [20], ok_table) == B.HAT_ERR_OUT_OF_RANGE
+    assert _status(_plan, c, [10], [20], [[0, 64, 2, 3]]) == B.HAT_ERR_OUT_OF_RANGE
+    assert _status(_plan, c, [10], [20], [[0, -1, 2, 3]]) == B.HAT_ERR_OUT_OF_RANGE
+    assert _status(_plan, c, [10], [20], [[0, 1, -1, 9999]]) == B.HAT_OK
+    # a page written by two requests; reading a shared page is fine
+    assert _status(_plan, c, [0, 0], [5, 5], [[7], [7]]) == B.HAT_ERR_OUT_OF_RANGE
+    assert _status(_plan, c, [16, 16], [5, 5], [[7, 8], [7, 9]]) == B.HAT_OK
+    # unsupported geometry
+    assert _status(_plan, _cache(page_size=32), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
+    assert _status(_plan, _cache(head_dim=96), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
+    assert _status(_plan, _cache(dtype=2), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
+    assert _status(_plan, _cache(stride_token=132), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
+    assert _status(_plan, c, [0], [4], [[0]], H=8) == B.HAT_ERR_UNSUPPORTED       # q heads != kv heads
+    # null descriptors
+    out = C.c_void_p()
+    assert hat_lib.hat_plan_create(None, None, C.byref(out)) == B.HAT_ERR_INVALID_ARG
+    assert hat_lib.hat_plan_create(C.byref(c), None, None) == B.HAT_ERR_INVALID_ARG
+    assert hat_lib.hat_plan_destroy(None) == B.HAT_OK
+
+
+def test_empty_batches_are_valid(hat_lib):
+    c = _cache()
+    p = _plan(c, [], [], np.zeros((0, 0), np.int32))
+    assert B.hat_plan_get_info(p).total_rows == 0
+    p = _plan(c, [5, 0], [0, 0], [[0], [1]])
+    info = B.hat_plan_get_info(p).as_dict()
+    assert info["total_rows"] == 0 and info["num_verify_items"] == 0 and info["workspace_bytes"] == 0
+
+
+def test_host_only_plan_cannot_launch(hat_lib):
+    c = _cache()
+    p = _plan(c, [10], [4], [[0]])
+    assert hat_lib.hat_kv_append(C.byref(c), p.handle, None, None, None) == B.HAT_ERR_INVALID_ARG
+
+
+def _info(sc, step=0, **env):
+    st = sc.steps[step]
+    spec = sc.cache
+    c = B.make_cache_desc(spec.dtype, spec.num_pages, spec.num_heads, spec.head_dim, spec.stride_page,
+                          spec.stride_token, spec.stride_head)
+    p = B.hat_plan_create(c, spec.num_heads, st.cu_chunk, st.prefix_len, st.chunk_len, st.block_table,
+                          B.HAT_PLAN_HOST_ONLY)
+    return B.hat_plan_get_info(p).as_dict()
+
+
+def _shapes_only(maker, **kw):
+    """Scenario with 1 head x 64 so that building it is cheap; shapes are what matters here."""
+    return maker(H=1, d=64, **kw)
+
+
+def test_schedule_of_the_verify_batch(hat_lib):
+    sc = _shapes_only(W.spec_verify)
+    st = sc.steps[0]
+    info = _info(sc)
+    assert info["num_verify_requests"] == 30 and info["num_prefill_requests"] == 0
+    assert info["max_splits"] <= 32
+    L = info["verify_split_len"]
+    assert L % 16 == 0 and L >= 16
+    def pieces(n):                       # ranges of L keys, lengthened so that no request has more than 32
+        per = max(L, -(-(-(-n // 32)) // 16) * 16)
+        return -(-n // per)
+    want_items = sum(pieces(int(p + c)) for p, c in zip(st.prefix_len, st.chunk_len))
+    assert info["num_verify_items"] == want_items
+    split_rows = sum(int(c) for p, c in zip(st.prefix_len, st.chunk_len) if pieces(int(p + c)) > 1)
+    assert info["num_merge_rows"] == split_rows
+    # flops and bytes follow the stated conventions
+    d, H = 64, 1
+    F = sum(4 * d * H * (int(c) * int(p) + int(c) * (int(c) + 1) // 2) for p, c in zip(st.prefix_len, st.chunk_len))
+    Bk = sum(2 * (int(p) + int(c)) * H * d * 2 for p, c in zip(st.prefix_len, st.chunk_len))
+    assert info["attn_flops"] == F and info["kv_read_bytes"] == Bk
+
+
+def test_schedule_of_prefill_and_mixed_batches(hat_lib):
+    sc = _shapes_only(W.ragged_prefill)
+    st = sc.steps[0]
+    info = _info(sc)
+    assert info["num_prefill_requests"] == 30 and info["num_verify_requests"] == 0
+    rows = info["prefill_tile_rows"]
+    tiles = sum(-(-int(c) // rows) for c in st.chunk_len)
+    assert info["num_prefill_items"] >= tiles
+    sc = _shapes_only(W.mixed_13b)
+    info = _info(sc)
+    assert info["num_prefill_requests"] == 8 and info["num_verify_requests"] == 32
+    assert info["total_rows"] == 8 * 512 + 32 * 4
+    assert info["max_splits"] <= 32
+
+
+def test_long_request_never_exceeds_32_key_ranges(hat_lib):
+    c = _cache(num_pages=4096)
+    n = 60000
+    table = [list(range((n + 4 + 15) // 16))]
+    p = _plan(c, [n], [4], table)
+    info = B.hat_plan_get_info(p).as_dict()
+    assert info["max_splits"] <= 32 and info["num_verify_items"] == info["max_splits"]

@@ -1,0 +1,258 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element on reduced
+sizes of the five workloads, on sampled rows at their full sizes, and on the edge cases."""
+import types
+
+import numpy as np
+import pytest
+
+from oracle import hat_oracle as O
+from paper_2503_18989_b200 import workloads as W
+
+from common import assert_parity, oracle_replay
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(sc, device, fused_append=True):
+    from paper_2503_18989_b200 import runner
+    return runner.run_scenario(sc, device, fused_append=fused_append)
+
+
+def _check_full(sc, device, fused_append=True):
+    """Every element of out/lse of every step, and both pools bit for bit."""
+    cache, got = _run(sc, device, fused_append)
+    kp, vp, want = oracle_replay(sc)
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, kp), "K pool differs from the oracle's append"
+    assert np.array_equal(gv, vp), "V pool differs from the oracle's append"
+    for s, ((go, gl), (wo, wl)) in enumerate(zip(got, want)):
+        assert_parity(go, wo, f"{sc.name} step {s} out")
+        assert_parity(gl, wl, f"{sc.name} step {s} lse")
+    return got, want
+
+
+def _check_sampled(sc, device, num_samples=400, seed=0):
+    """Full-size run: pools bit for bit; out/lse on sampled (request, row, head) triples, always
+    including the first and last row of every request."""
+    cache, got = _run(sc, device)
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    rng = np.random.default_rng(seed)
+    for s, st in enumerate(sc.steps):
+        O.kv_append(sc.cache, kp, vp, st)
+        samples = []
+        live = [r for r in range(st.num_requests) if st.chunk_len[r] > 0]
+        for r in live:
+            for i in {0, int(st.chunk_len[r]) - 1}:
+                samples.append((r, i, int(rng.integers(sc.cache.num_heads))))
+        while len(samples) < num_samples // len(sc.steps):
+            r = live[int(rng.integers(len(live)))]
+            samples.append((r, int(rng.integers(st.chunk_len[r])), int(rng.integers(sc.cache.num_heads))))
+        samples = np.asarray(samples, np.int64)
+        wo, wl = O.attention_rows(sc.cache, kp, vp, st, samples)
+        rows = st.cu_chunk[samples[:, 0]] + samples[:, 1]
+        go = got[s][0][rows, samples[:, 2]]
+        gl = got[s][1][rows, samples[:, 2]]
+        assert_parity(go, wo, f"{sc.name} step {s} sampled out")
+        assert_parity(gl, wl, f"{sc.name} step {s} sampled lse")
+        assert np.isfinite(got[s][0]).all() and np.isfinite(got[s][1]).all()
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+
+
+# ----------------------------------------------------------------------------
+# the five workloads: reduced sizes, every element
+# ----------------------------------------------------------------------------
+def test_tiny_every_element(cuda_device):
+    _check_full(W.tiny(), cuda_device)                       # the full "tiny" configuration
+
+
+def test_llama7b_chunked_reduced(cuda_device):
+    _check_full(W.llama7b_chunked(prompt=640, chunk=256, H=4), cuda_device)   # 256, 256, ragged 128
+
+
+def test_ragged_prefill_reduced(cuda_device):
+    _check_full(W.ragged_prefill(num_requests=7, max_prefix=640, H=3), cuda_device)
+
+
+def test_spec_verify_reduced(cuda_device):
+    _check_full(W.spec_verify(num_requests=9, min_prefix=100, max_prefix=1500, H=5), cuda_device)
+
+
+def test_mixed_13b_reduced(cuda_device):
+    _check_full(W.mixed_13b(num_prefill=2, prefill_chunk=512, max_prefill_prefix=700, num_verify=6,
+                            min_verify_prefix=200, max_verify_prefix=1200, H=3), cuda_device)
+
+
+# ----------------------------------------------------------------------------
+# the five workloads: full sizes, sampled rows
+# ----------------------------------------------------------------------------
+def test_llama7b_chunked_full_size_sampled(cuda_device):
+    _check_sampled(W.llama7b_chunked(), cuda_device, num_samples=480)
+
+
+def test_ragged_prefill_full_size_sampled(cuda_device):
+    _check_sampled(W.ragged_prefill(), cuda_device)
+
+
+def test_spec_verify_full_size_sampled(cuda_device):
+    _check_sampled(W.spec_verify(), cuda_device)
+
+
+def test_mixed_13b_full_size_sampled(cuda_device):
+    _check_sampled(W.mixed_13b(), cuda_device)
+
+
+# ----------------------------------------------------------------------------
+# variants and edge cases
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,layout", [("bf16", 128, "paged"), ("fp16", 64, "paged"), ("bf16", 64, "contiguous"),
+                                           ("fp16", 128, "contiguous")])
+def test_dtype_headdim_layout_variants(cuda_device, dtype, d, layout):
+    sc = W.ragged_prefill(num_requests=4, max_prefix=300, chunk_choices=(17, 40, 64, 130), H=2, d=d, dtype=dtype,
+                          seed=77)
+    if layout == "contiguous":
+        sc.cache.layout = "contiguous"                       # same pool bits, different strides
+    _check_full(sc, cuda_device)
+    sc = W.spec_verify(num_requests=4, min_prefix=1, max_prefix=400, max_draft=16, H=2, d=d, dtype=dtype, seed=78)
+    if layout == "contiguous":
+        sc.cache.layout = "contiguous"
+    _check_full(sc, cuda_device)
+
+
+def _manual(dtype, H, d, prefix, chunk, seed, num_pages=None, table=None, layout="paged"):
+    """Batch with hand-picked prefix/chunk lengths."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    if table is None:
+        table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=5)
+    st = W._make_step(seed + 100, dtype, H, d, prefix, chunk, table)
+    return W._scenario("manual", dtype, H, d, layout, num_pages, [st], seed + 100)
+
+
+def test_every_chunk_length_class_and_ragged_tails(cuda_device):
+    # 0 (no-op), 1 at an empty cache, 8, 16 (largest streaming), 17 (smallest tile), one short of and one past
+    # a tile, prefix not a multiple of the page size for a tile-class chunk
+    prefix = [40, 0, 33, 250, 5, 100, 77, 0, 1023]
+    chunk = [0, 1, 8, 16, 17, 63, 65, 129, 7]
+    _check_full(_manual("fp16", 2, 128, prefix, chunk, 5), cuda_device)
+    _check_full(_manual("bf16", 2, 64, prefix, chunk, 6), cuda_device)
+
+
+def test_empty_batch_and_all_zero_chunks(cuda_device):
+    from paper_2503_18989_b200 import binding as B, runner
+    sc = _manual("fp16", 2, 128, [10, 20], [0, 0], 9)
+    cache, got = _run(sc, cuda_device)
+    assert got[0][0].shape == (0, 2, 128)
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, sc.k_pool) and np.array_equal(gv, sc.v_pool)
+    plan = B.hat_plan_create(cache.desc, 2, np.zeros(1, np.int32), np.zeros(0, np.int32), np.zeros(0, np.int32),
+                             np.zeros((0, 0), np.int32))
+    B.hat_chunk_attention(cache.desc, plan, None, None, None, None, None)      # valid no-op
+    B.hat_kv_append(cache.desc, plan, None, None)
+
+
+def test_separate_append_equals_fused_append(cuda_device):
+    sc = W.mixed_13b(num_prefill=1, prefill_chunk=96, max_prefill_prefix=200, num_verify=3, min_verify_prefix=20,
+                     max_verify_prefix=300, H=2, seed=31)
+    c1, r1 = _run(sc, cuda_device, fused_append=True)
+    c2, r2 = _run(sc, cuda_device, fused_append=False)
+    for a, b in zip(c1.pools_to_host(), c2.pools_to_host()):
+        assert np.array_equal(a, b)
+    assert np.array_equal(r1[0][0], r2[0][0]) and np.array_equal(r1[0][1], r2[0][1])
+    # and running the same call twice gives the same bits
+    c3, r3 = _run(sc, cuda_device, fused_append=True)
+    assert np.array_equal(r1[0][0], r3[0][0]) and np.array_equal(r1[0][1], r3[0][1])
+
+
+def test_many_key_ranges_per_request(cuda_device):
+    # one long request alone in the batch: the scheduler cuts it into the maximum number of ranges
+    sc = _manual("fp16", 1, 128, [9000], [3], 12)
+    from paper_2503_18989_b200 import binding as B
+    got, want = _check_full(sc, cuda_device)
+
+
+def test_rollback_then_verify_again(cuda_device):
+    # Sec. 3.4: 6 drafts sent, 2 accepted; the next round restarts at prefix+2 and overwrites the rest.
+    H, d, P = 2, 128, 45
+    rng = np.random.Generator(np.random.PCG64(3))
+    table, num_pages = W._place_pages(rng, [P + 20], slack_pages=3)
+    s1 = W._make_step(500, "fp16", H, d, [P], [6], table)
+    s2 = W._make_step(600, "fp16", H, d, [P + 2], [5], table)
+    sc = W._scenario("rollback", "fp16", H, d, "paged", num_pages, [s1, s2], 700)
+    _check_full(sc, cuda_device)
+
+
+def test_explicit_scale_and_stale_nan_slots(cuda_device):
+    from paper_2503_18989_b200 import runner
+    sc = _manual("fp16", 2, 128, [37, 200], [4, 70], 15)
+    st = sc.steps[0]
+    # poison every slot the batch must not read: beyond prefix+chunk in the last page, and unowned pages
+    owned = np.zeros(sc.cache.num_pages, bool)
+    K = sc.k_pool.reshape(sc.cache.num_pages, 2, 16, 128); V = sc.v_pool.reshape(K.shape)
+    for r in range(2):
+        n = int(st.prefix_len[r] + st.chunk_len[r])
+        pages = st.block_table[r][: (n + 15) // 16]
+        owned[pages] = True
+        if n % 16:
+            K[pages[-1], :, n % 16:, :] = 0x7E00           # fp16 NaN
+            V[pages[-1], :, n % 16:, :] = 0x7E00
+    K[~owned] = 0x7E00; V[~owned] = 0x7E00
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    ds.attend(fused_append=True, sm_scale=0.05)
+    go, gl = ds.results()
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(sc.cache, kp, vp, st)
+    wo, wl = O.chunk_attention(sc.cache, kp, vp, st, sm_scale=float(np.float32(0.05)))
+    assert_parity(go, wo, "scaled out"); assert_parity(gl, wl, "scaled lse")
+
+
+def test_launch_errors_are_reported_before_any_work(cuda_device):
+    from paper_2503_18989_b200 import binding as B, runner
+    sc = W.spec_verify(num_requests=2, min_prefix=600, max_prefix=900, H=2, seed=41)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert ds.workspace_bytes > 0
+    with pytest.raises(B.HatError) as e:
+        B.hat_chunk_attention(cache.desc, ds.plan, ds.q, None, None, ds.out, ds.lse, 0.0, ds.workspace, 16)
+    assert e.value.status == B.HAT_ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(B.HatError) as e:
+        B.hat_chunk_attention(cache.desc, ds.plan, ds.q, ds.k_new, None, ds.out, ds.lse, 0.0, ds.workspace,
+                              ds.workspace_bytes)
+    assert e.value.status == B.HAT_ERR_INVALID_ARG
+    with pytest.raises(B.HatError) as e:
+        B.hat_chunk_attention(cache.desc, ds.plan, None, None, None, ds.out, ds.lse, 0.0, ds.workspace,
+                              ds.workspace_bytes)
+    assert e.value.status == B.HAT_ERR_INVALID_ARG
+    other = B.make_cache_desc("bf16", sc.cache.num_pages, 2, 128, sc.cache.stride_page, sc.cache.stride_token,
+                              sc.cache.stride_head, cache.k, cache.v)
+    with pytest.raises(B.HatError) as e:
+        B.hat_kv_append(other, ds.plan, ds.k_new, ds.v_new)
+    assert e.value.status == B.HAT_ERR_INVALID_ARG
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, sc.k_pool) and np.array_equal(gv, sc.v_pool)     # nothing was written
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+
+
+def test_host_buffer_entry_point(cuda_device):
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    sc = W.mixed_13b(num_prefill=1, prefill_chunk=80, max_prefill_prefix=150, num_verify=2, min_verify_prefix=30,
+                     max_verify_prefix=700, H=2, seed=51)
+    st = sc.steps[0]
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    T, H, d = st.total_rows, 2, 128
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    q, k, v = pin(st.q), pin(st.k_new), pin(st.v_new)
+    out = torch.empty((T, H, d), dtype=torch.float32).pin_memory()
+    lse = torch.empty((T, H), dtype=torch.float32).pin_memory()
+    nbytes = B.hat_plan_staging_bytes(ds.plan)
+    staging = torch.empty(nbytes, dtype=torch.uint8, device=cuda_device)
+    B.hat_chunk_attention_host(cache.desc, ds.plan, q, k, v, out, lse, 0.0, staging, nbytes, ds.workspace,
+                               ds.workspace_bytes)
+    torch.cuda.synchronize()
+    kp, vp, want = oracle_replay(sc)
+    assert_parity(out.numpy(), want[0][0], "host entry out")
+    assert_parity(lse.numpy(), want[0][1], "host entry lse")
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
