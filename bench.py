@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the chunk-attention hot path (plan -> KV append -> tile + streaming attention -> merge).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole path over one synthetic batch: one hat_chunk_attention call with the
+append fused (for the multi-call workloads, the whole sequence of calls).  Prints ONE JSON line.
+With N > 1 (torchrun) every rank runs an independent replica of the batch (the path has no
+inter-GPU exchange); time is the maximum over ranks and the value sums the work of all ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_18989_b200 import workloads as W  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+VERIFY_MAX_ROWS = 16          # chunks up to this length take the streaming kernel
+SLOT_NAMES = ["kv_append", "tile_attention", "streaming_attention", "merge"]
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"]))}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------
+# algorithmic work of a batch (conventions: only unmasked (q,k) pairs, 2d flop for QK^T + 2d for PV;
+# every visible K and V row read once per head)
+# ----------------------------------------------------------------------------
+def step_work(cache, st):
+    H, d, e = cache.num_heads, cache.head_dim, 2
+    P = st.prefix_len.astype(np.int64)
+    Cn = st.chunk_len.astype(np.int64)
+    pairs = Cn * P + Cn * (Cn + 1) // 2
+    flops = 4 * d * H * pairs
+    kv_bytes = 2 * (P + Cn) * H * d * e * (Cn > 0)
+    io_bytes = Cn * H * d * e + Cn * H * d * 4 + Cn * H * 4            # q in, out + lse out
+    short = (Cn > 0) & (Cn <= VERIFY_MAX_ROWS)
+    long_ = Cn > VERIFY_MAX_ROWS
+    T = int(Cn.sum())
+    return {
+        "flops": int(flops.sum()),
+        "tile_flops": int(flops[long_].sum()), "tile_bytes": int((kv_bytes + io_bytes)[long_].sum()),
+        "stream_flops": int(flops[short].sum()), "stream_bytes": int((kv_bytes + io_bytes)[short].sum()),
+        "append_bytes": int(4 * T * H * d * e),
+        "kv_bytes": int(kv_bytes.sum()),
+        "rows": T,
+    }
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.samples = []
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        threading.Thread(target=self._pump, daemon=True).start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0, t1):
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        pool = inside or self.samples[-3:]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for _, line in pool:
+            f = [x.strip() for x in line.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except Exception:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(inside)}
+
+
+def pick_oracle_sample(cache, st, rng, target_flops):
+    """(request, row, head) units drawn uniformly over all (row, head) pairs until ~target_flops."""
+    H, d = cache.num_heads, cache.head_dim
+    live = np.nonzero(st.chunk_len > 0)[0]
+    rows_req = np.repeat(live, st.chunk_len[live])
+    rows_i = np.concatenate([np.arange(int(st.chunk_len[r])) for r in live])
+    units, flops = [], 0
+    while flops < target_flops and len(units) < 200000:
+        t = int(rng.integers(len(rows_req)))
+        r, i, h = int(rows_req[t]), int(rows_i[t]), int(rng.integers(H))
+        units.append((r, i, h))
+        flops += 4 * d * (int(st.prefix_len[r]) + i + 1)
+    return np.asarray(units, np.int64), flops
+
+
+def time_oracle(sc, budget_s, seed=0):
+    """The CPU oracle on a bounded sample of the last call of the workload.  Returns
+    (flop/s, cores, description, units, flops_per_run)."""
+    from oracle import hat_oracle as O
+    st = sc.steps[-1]
+    kp, vp = sc.k_pool, sc.v_pool
+    for s in sc.steps:                       # the oracle needs the chunk's K/V in its pool (append, then attend)
+        O.kv_append(sc.cache, kp, vp, s)
+    rng = np.random.default_rng(seed)
+    units, fl = pick_oracle_sample(sc.cache, st, rng, 2e8)
+    t0 = time.perf_counter(); O.attention_rows(sc.cache, kp, vp, st, units); dt = time.perf_counter() - t0
+    rate = fl / max(dt, 1e-6)
+    units, fl = pick_oracle_sample(sc.cache, st, rng, rate * budget_s)
+    t0 = time.perf_counter(); O.attention_rows(sc.cache, kp, vp, st, units); dt = time.perf_counter() - t0
+    return fl / dt, O.threads(), f"{len(units)} (request,row,head) units of the batch, {fl:.3g} flop, {dt:.1f} s", \
+        units, fl
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle, as it stands, on the host cores."""
+    if rank != 0:
+        return
+    from oracle import hat_oracle as O
+    sc = W.WORKLOADS[args.workload]()
+    st = sc.steps[-1]
+    for s in sc.steps:
+        O.kv_append(sc.cache, sc.k_pool, sc.v_pool, s)
+    rng = np.random.default_rng(0)
+    units, fl = pick_oracle_sample(sc.cache, st, rng, 2e8)
+    t0 = time.perf_counter(); O.attention_rows(sc.cache, sc.k_pool, sc.v_pool, st, units)
+    rate = fl / max(time.perf_counter() - t0, 1e-6)
+    per_step = min(20.0, 150.0 / max(1, args.steps + args.warmup))
+    units, fl = pick_oracle_sample(sc.cache, st, rng, rate * per_step)
+    for _ in range(args.warmup):
+        O.attention_rows(sc.cache, sc.k_pool, sc.v_pool, st, units)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.attention_rows(sc.cache, sc.k_pool, sc.v_pool, st, units)
+    dt = time.perf_counter() - t0
+    value = fl * args.steps / dt / 1e12
+    sample = f"{len(units)} (request,row,head) units per step ({fl:.3g} flop) of workload {sc.name}"
+    print(json.dumps({
+        "impl": "reference", "metric": "chunk_attention_tflops", "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": sc.name, "note": "CPU oracle on a bounded sample of the batch per step"},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": O.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="mixed_13b", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if args.steps is None:
+            args.steps = 5
+        if args.warmup is None:
+            args.warmup = 1
+        run_reference(args, rank)
+        return
+    if args.steps is None:
+        args.steps = 1000 if args.workload in ("mixed_13b", "ragged_prefill", "spec_verify") else 200
+    if args.warmup is None:
+        args.warmup = 20
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2503_18989_b200 import binding as B
+    from paper_2503_18989_b200 import build as hat_build
+    from paper_2503_18989_b200 import runner
+
+    if rank == 0:
+        hat_build.build()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+        dist.barrier()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    peaks, peak_kind = load_peaks()
+
+    # ---- inputs: one replica of the batch per rank (seeded; different values per rank)
+    sc = W.WORKLOADS[args.workload](seed=W.SEED_BASE + list(W.WORKLOADS).index(args.workload) + 1 + 1000 * rank)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, device)
+    steps = [runner.DeviceStep(cache, st) for st in sc.steps]
+    works = [step_work(sc.cache, st) for st in sc.steps]
+    total = {k: sum(w[k] for w in works) for k in works[0]}
+    kv_resident = 2 * sc.k_pool.nbytes
+    flush_l2 = total["kv_bytes"] / len(sc.steps) < 2 * L2_BYTES
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device) if flush_l2 else None
+    stream = torch.cuda.current_stream(device).cuda_stream
+
+    def one_step():
+        for ds in steps:
+            ds.attend(fused_append=True, stream=stream)
+
+    for _ in range(args.warmup):
+        one_step()
+    torch.cuda.synchronize(device)
+    for ds in steps:
+        if B.hat_last_device_status(ds.plan, stream) != B.HAT_OK:
+            raise RuntimeError("device-side wait timed out during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+
+    # ---- timed region: exactly K steps, device events, per-kernel events recorded by the library
+    K = args.steps
+    for ds in steps:
+        B.hat_plan_enable_timing(ds.plan, K)
+    launches0 = B.hat_launch_count()
+    barrier(); torch.cuda.synchronize(device)
+    t_wall0 = time.time()
+    if not flush_l2:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            one_step()
+        e1.record()
+        torch.cuda.synchronize(device)
+        elapsed_ms = e0.elapsed_time(e1)
+    else:
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for a, b in evs:
+            flush_buf.zero_()                 # evict the KV working set from L2 (not timed)
+            a.record(); one_step(); b.record()
+        torch.cuda.synchronize(device)
+        elapsed_ms = sum(a.elapsed_time(b) for a, b in evs)
+    t_wall1 = time.time()
+    barrier()
+    launches = B.hat_launch_count() - launches0
+    kernel_ms = np.zeros(B.HAT_TIMING_SLOTS)
+    kernel_calls = np.zeros(B.HAT_TIMING_SLOTS)
+    for ds in steps:
+        ms = B.hat_plan_read_timing(ds.plan, K)
+        kernel_ms += ms.sum(axis=0)
+        kernel_calls += (ms > 0).sum(axis=0)
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    # ---- end to end through the host-buffer entry point: H2D of q/k_new/v_new and D2H of out/lse per step
+    Ke = max(1, min(K, 100))
+    host = []
+    for ds, st in zip(steps, sc.steps):
+        T, H, d = st.total_rows, sc.cache.num_heads, sc.cache.head_dim
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        nb = B.hat_plan_staging_bytes(ds.plan)
+        host.append((pin(st.q), pin(st.k_new), pin(st.v_new),
+                     torch.empty((T, H, d), dtype=torch.float32).pin_memory(),
+                     torch.empty((T, H), dtype=torch.float32).pin_memory(),
+                     torch.empty(max(nb, 256), dtype=torch.uint8, device=device), nb))
+
+    def one_step_host():
+        for ds, (q, k, v, o, l, stg, nb) in zip(steps, host):
+            B.hat_chunk_attention_host(cache.desc, ds.plan, q, k, v, o, l, 0.0, stg, nb, ds.workspace,
+                                       ds.workspace_bytes, stream)
+    for _ in range(3):
+        one_step_host()
+    barrier(); torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(Ke):
+        one_step_host()
+    e1.record()
+    torch.cuda.synchronize(device)
+    e2e_ms = e0.elapsed_time(e1)
+    barrier()
+    sampler.stop()
+    h2d = sum(3 * st.q.nbytes for st in sc.steps)
+    d2h = sum(st.total_rows * sc.cache.num_heads * (sc.cache.head_dim + 1) * 4 for st in sc.steps)
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        ms_per_step = elapsed_ms / K
+        value = world * total["flops"] / (ms_per_step * 1e-3) / 1e12
+        e2e_value = world * total["flops"] / (e2e_ms / Ke * 1e-3) / 1e12
+
+        # per-kernel achieved throughput against its roofline
+        avg = np.where(kernel_calls > 0, kernel_ms / np.maximum(kernel_calls, 1), 0.0)   # ms per launch
+        per_launch = {
+            "kv_append": ("hbm", total["append_bytes"] / len(sc.steps)),
+            "tile_attention": ("tensor", total["tile_flops"] / max(1, sum(1 for w in works if w["tile_flops"]))),
+            "streaming_attention": ("hbm", total["stream_bytes"] / max(1, sum(1 for w in works if w["stream_bytes"]))),
+            "merge": ("hbm", 0.0),
+        }
+        tensor_peak = peaks["bf16_tflops_sustained"]
+        kernels = {}
+        for i, name in enumerate(SLOT_NAMES):
+            if kernel_calls[i] == 0:
+                continue
+            bound, alg = per_launch[name]
+            sec = avg[i] * 1e-3
+            if bound == "tensor":
+                ach, peak, unit = alg / sec / 1e12, tensor_peak, "TFLOP/s"
+            else:
+                ach, peak, unit = alg / sec / 1e9, peaks["hbm_gbs"], "GB/s"
+            kernels[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                             "ms_per_launch": float(avg[i]), "launches": int(kernel_calls[i]),
+                             "share": float(kernel_ms[i] / max(kernel_ms.sum(), 1e-9))}
+        dominant = max(kernels, key=lambda n: kernels[n]["share"])
+        roof = {k: kernels[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
+        roof.update({"kernel": dominant, "traffic": None, "peak_source": f"{peak_kind} "
+                     + ("bf16 sustained" if roof["bound"] == "tensor" else "HBM copy")})
+        # the tile kernel against the memory roofline as well (short chunks are HBM-bound)
+        if "tile_attention" in kernels:
+            sec = kernels["tile_attention"]["ms_per_launch"] * 1e-3
+            n_tile_calls = max(1, sum(1 for w in works if w["tile_flops"]))
+            kernels["tile_attention"]["hbm_gbs"] = total["tile_bytes"] / n_tile_calls / sec / 1e9
+            kernels["tile_attention"]["hbm_frac"] = kernels["tile_attention"]["hbm_gbs"] / peaks["hbm_gbs"]
+
+        line = {
+            "metric": "chunk_attention_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": K, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": sc.cache.dtype + " in, f32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": sc.name, "requests": int(sc.steps[-1].num_requests), "rows": total["rows"],
+                       "heads": sc.cache.num_heads, "head_dim": sc.cache.head_dim, "page_size": 16,
+                       "calls_per_step": len(sc.steps), "kv_resident_bytes": int(kv_resident),
+                       "l2": "flushed between steps" if flush_l2 else "KV working set larger than L2",
+                       "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(d2h), "steps": Ke, "ms_per_step": e2e_ms / Ke},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roof,
+            "kernels": kernels,
+            "kv_gbs": world * total["kv_bytes"] / (ms_per_step * 1e-3) / 1e9,
+            "plan": steps[-1].info,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            rate, cores, sample, _, _ = time_oracle(sc, args.cpu_budget)
+            line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                                    "sample": sample}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

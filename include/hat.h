@@ -200,6 +200,23 @@ int hat_chunk_attention_host(const hat_cache_desc* cache, const hat_plan* plan,
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Optional per-kernel timing for benchmarks (not part of the method).  After
+ * hat_plan_enable_timing, each of the next max_calls calls of
+ * hat_chunk_attention / hat_chunk_attention_host on this plan records CUDA
+ * events on its stream around each kernel it launches (this creates
+ * 5*max_calls events once, here, not in the attention call).
+ * hat_plan_read_timing waits for the recorded events and writes, per recorded
+ * call, HAT_TIMING_SLOTS durations in milliseconds: [0] KV append, [1] tile
+ * (prefill-class) attention, [2] streaming (verify-class) attention, [3] merge;
+ * 0 where a kernel was not launched.  It then rewinds the recorder.
+ *   ms          host, [capacity_calls][HAT_TIMING_SLOTS]
+ *   num_calls   host, out: calls written
+ */
+#define HAT_TIMING_SLOTS 4
+int hat_plan_enable_timing(hat_plan* plan, int max_calls);
+int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num_calls);
+
+/*
  * Read the device-side status word of a plan (synchronises `stream`).  *out is
  * HAT_OK, or HAT_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up
  * since the plan was created; results of such a call are undefined.

@@ -33,8 +33,9 @@ EXPORTS = [
     "hat_status_string", "hat_version", "hat_last_cuda_error", "hat_launch_count",
     "hat_plan_create", "hat_plan_get_info", "hat_plan_workspace_bytes", "hat_plan_destroy",
     "hat_kv_append", "hat_chunk_attention", "hat_plan_staging_bytes", "hat_chunk_attention_host",
-    "hat_last_device_status",
+    "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
 ]
+HAT_TIMING_SLOTS = 4
 
 
 class hat_cache_desc(C.Structure):
@@ -110,6 +111,10 @@ def lib() -> C.CDLL:
                                                vp, sz, vp, sz, vp]
         L.hat_last_device_status.restype = i32
         L.hat_last_device_status.argtypes = [vp, vp, C.POINTER(i32)]
+        L.hat_plan_enable_timing.restype = i32
+        L.hat_plan_enable_timing.argtypes = [vp, i32]
+        L.hat_plan_read_timing.restype = i32
+        L.hat_plan_read_timing.argtypes = [vp, vp, i32, C.POINTER(i32)]
         _lib = L
     return _lib
 
@@ -238,3 +243,15 @@ def hat_last_device_status(plan, stream: int = 0) -> int:
     st = C.c_int()
     _check(lib().hat_last_device_status(_h(plan), stream or None, C.byref(st)), "hat_last_device_status")
     return int(st.value)
+
+
+def hat_plan_enable_timing(plan, max_calls: int) -> None:
+    _check(lib().hat_plan_enable_timing(_h(plan), int(max_calls)), "hat_plan_enable_timing")
+
+
+def hat_plan_read_timing(plan, capacity_calls: int) -> np.ndarray:
+    """Per recorded call: milliseconds of [append, tile attention, streaming attention, merge]."""
+    ms = np.zeros((int(capacity_calls), HAT_TIMING_SLOTS), dtype=np.float32)
+    n = C.c_int()
+    _check(lib().hat_plan_read_timing(_h(plan), _ptr(ms), int(capacity_calls), C.byref(n)), "hat_plan_read_timing")
+    return ms[: n.value]

@@ -51,10 +51,12 @@ struct Mma<__half> {
             : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
             : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
     }
+    static constexpr bool kSplitP = false;
     static __device__ __forceinline__ uint32_t pack(float lo, float hi) {
         __half2 v = __floats2half2_rn(lo, hi);
         return *reinterpret_cast<uint32_t*>(&v);
     }
+    static __device__ __forceinline__ uint32_t pack_residual(float, float, uint32_t) { return 0u; }
 };
 template <>
 struct Mma<__nv_bfloat16> {
@@ -64,9 +66,15 @@ struct Mma<__nv_bfloat16> {
             : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
             : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
     }
+    static constexpr bool kSplitP = true;
     static __device__ __forceinline__ uint32_t pack(float lo, float hi) {
         __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
         return *reinterpret_cast<uint32_t*>(&v);
+    }
+    // what the rounding in pack() dropped: (lo, hi) minus the packed pair, itself rounded to bf16
+    static __device__ __forceinline__ uint32_t pack_residual(float lo, float hi, uint32_t packed) {
+        const float plo = __uint_as_float(packed << 16), phi = __uint_as_float(packed & 0xffff0000u);
+        return pack(lo - plo, hi - phi);
     }
 };
 
@@ -253,11 +261,18 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
         // O += P V
 #pragma unroll
         for (int kp = 0; kp < KB / 16; ++kp) {
-            uint32_t pa[4];
+            uint32_t pa[4], pl[4];
             pa[0] = Mma<T>::pack(s[2 * kp][0], s[2 * kp][1]);
             pa[1] = Mma<T>::pack(s[2 * kp][2], s[2 * kp][3]);
             pa[2] = Mma<T>::pack(s[2 * kp + 1][0], s[2 * kp + 1][1]);
             pa[3] = Mma<T>::pack(s[2 * kp + 1][2], s[2 * kp + 1][3]);
+            if constexpr (Mma<T>::kSplitP) {
+                // bf16 keeps 8 significant bits: carry the rounding remainder of P in a second operand
+                pl[0] = Mma<T>::pack_residual(s[2 * kp][0], s[2 * kp][1], pa[0]);
+                pl[1] = Mma<T>::pack_residual(s[2 * kp][2], s[2 * kp][3], pa[1]);
+                pl[2] = Mma<T>::pack_residual(s[2 * kp + 1][0], s[2 * kp + 1][1], pa[2]);
+                pl[3] = Mma<T>::pack_residual(s[2 * kp + 1][2], s[2 * kp + 1][3], pa[3]);
+            }
 #pragma unroll
             for (int dn = 0; dn < D / 16; ++dn) {
                 const int mi = lane >> 3;
@@ -266,6 +281,10 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
                 ldmatrix_x4_trans(b0, b1, b2, b3, vst + swz<D>(key, dn * 2 + (mi >> 1)));
                 Mma<T>::run(o[2 * dn], pa, b0, b1);
                 Mma<T>::run(o[2 * dn + 1], pa, b2, b3);
+                if constexpr (Mma<T>::kSplitP) {
+                    Mma<T>::run(o[2 * dn], pl, b0, b1);
+                    Mma<T>::run(o[2 * dn + 1], pl, b2, b3);
+                }
             }
         }
     }

@@ -119,8 +119,8 @@ static void schedule(hat_plan* p, int num_sms) {
         const int64_t want_ctas = (int64_t)num_sms * 2;
         if (tiles > 0 && tiles * H < want_ctas) {
             // aim for want_ctas pieces of equal length, not shorter than 256 keys
-            int64_t pieces = ceil_div((int)want_ctas, H);
-            psplit = std::max<int64_t>(256, round_up((int)ceil_div((int)tile_keys, (int)pieces), 64));
+            const int pieces = ceil_div((int)want_ctas, H);
+            psplit = std::max(256, round_up((int)((tile_keys + pieces - 1) / pieces), 64));
         }
     }
     if (psplit > 0) psplit = round_up(psplit, 64);
@@ -152,7 +152,7 @@ static void schedule(hat_plan* p, int num_sms) {
     info.num_prefill_items = (int32_t)p->prefill_items.size();
     info.num_merge_rows = (int32_t)p->merge_rows.size();
     const int64_t d = p->head_dim;
-    int64_t part_out_bytes = round_up((int)0, 1) + p->part_rows * H * d * 4;
+    int64_t part_out_bytes = p->part_rows * H * d * 4;
     part_out_bytes = (part_out_bytes + 255) / 256 * 256;
     info.workspace_bytes = p->part_rows ? part_out_bytes + ((p->part_rows * H * 4 + 255) / 256 * 256) : 0;
 }
@@ -296,6 +296,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->device = -1;
     p->part_rows = 0;
     p->dev_blob = nullptr;
+    p->timing = nullptr;
     std::memset(&p->info, 0, sizeof p->info);
     std::memset(&p->dev, 0, sizeof p->dev);
     p->cu_chunk.assign(batch->cu_chunk, batch->cu_chunk + R + 1);
@@ -349,6 +350,10 @@ int hat_plan_workspace_bytes(const hat_plan* plan, size_t* out) {
 int hat_plan_destroy(hat_plan* plan) {
     if (!plan) return HAT_OK;
     int st = HAT_OK;
+    if (plan->timing) {
+        for (cudaEvent_t ev : plan->timing->events) cudaEventDestroy(ev);
+        delete plan->timing;
+    }
     if (plan->dev_blob) {
         cudaError_t e = cudaFree(plan->dev_blob);
         if (e != cudaSuccess) st = cuda_fail(e);
@@ -387,10 +392,23 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
+    // optional event recorder: slot boundaries 0..4 around append, tile, streaming, merge
+    Timing* tm = plan->timing;
+    int call = -1;
+    if (tm && tm->next < tm->max_calls) call = tm->next++;
+    auto mark = [&](int boundary) {
+        if (call >= 0) cudaEventRecord(tm->events[(size_t)call * 5 + boundary], s);
+    };
+    auto ran = [&](int slot) {
+        if (call >= 0) tm->launched[(size_t)call * HAT_TIMING_SLOTS + slot] = 1;
+    };
+    mark(0);
     if (k_new) {
         e = launch_kv_append(plan, view_of(cache), cache->k_pool, cache->v_pool, k_new, v_new, s);
         if (e != cudaSuccess) return cuda_fail(e);
+        ran(0);
     }
+    mark(1);
     AttnArgs a;
     a.plan = plan->dev;
     a.cache = view_of(cache);
@@ -406,15 +424,67 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
     if (!plan->prefill_items.empty()) {
         e = launch_attn_mma(plan, a, /*verify_class=*/false, s);
         if (e != cudaSuccess) return cuda_fail(e);
+        ran(1);
     }
+    mark(2);
     if (!plan->verify_items.empty()) {
         e = launch_attn_mma(plan, a, /*verify_class=*/true, s);
         if (e != cudaSuccess) return cuda_fail(e);
+        ran(2);
     }
+    mark(3);
     if (!plan->merge_rows.empty()) {
         e = launch_merge(plan, a, s);
         if (e != cudaSuccess) return cuda_fail(e);
+        ran(3);
     }
+    mark(4);
+    return HAT_OK;
+}
+
+int hat_plan_enable_timing(hat_plan* plan, int max_calls) {
+    if (!plan || plan->host_only || max_calls <= 0 || max_calls > (1 << 20)) return HAT_ERR_INVALID_ARG;
+    if (plan->timing) {
+        for (cudaEvent_t ev : plan->timing->events) cudaEventDestroy(ev);
+        delete plan->timing;
+        plan->timing = nullptr;
+    }
+    Timing* tm = new (std::nothrow) Timing();
+    if (!tm) return HAT_ERR_INVALID_ARG;
+    tm->events.resize((size_t)max_calls * 5);
+    for (size_t i = 0; i < tm->events.size(); ++i) {
+        cudaError_t e = cudaEventCreate(&tm->events[i]);
+        if (e != cudaSuccess) {
+            for (size_t j = 0; j < i; ++j) cudaEventDestroy(tm->events[j]);
+            delete tm;
+            return cuda_fail(e);
+        }
+    }
+    tm->launched.assign((size_t)max_calls * HAT_TIMING_SLOTS, 0);
+    tm->max_calls = max_calls;
+    plan->timing = tm;
+    return HAT_OK;
+}
+
+int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num_calls) {
+    if (!plan || !ms || !num_calls || capacity_calls < 0 || !plan->timing) return HAT_ERR_INVALID_ARG;
+    Timing* tm = plan->timing;
+    const int n = std::min(tm->next, capacity_calls);
+    for (int c = 0; c < n; ++c) {
+        cudaError_t e = cudaEventSynchronize(tm->events[(size_t)c * 5 + 4]);
+        if (e != cudaSuccess) return cuda_fail(e);
+        for (int sl = 0; sl < HAT_TIMING_SLOTS; ++sl) {
+            float t = 0.f;
+            if (tm->launched[(size_t)c * HAT_TIMING_SLOTS + sl]) {
+                e = cudaEventElapsedTime(&t, tm->events[(size_t)c * 5 + sl], tm->events[(size_t)c * 5 + sl + 1]);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
+            ms[(size_t)c * HAT_TIMING_SLOTS + sl] = t;
+        }
+    }
+    *num_calls = n;
+    tm->next = 0;
+    std::fill(tm->launched.begin(), tm->launched.end(), 0);
     return HAT_OK;
 }
 

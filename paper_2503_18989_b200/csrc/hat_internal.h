@@ -66,6 +66,16 @@ struct AttnArgs {
 
 }  // namespace hat
 
+namespace hat {
+// Event recorder for the optional per-kernel timing (5 events per recorded call).
+struct Timing {
+    std::vector<cudaEvent_t> events;
+    std::vector<uint8_t> launched;   // [call][slot]
+    int max_calls = 0;
+    int next = 0;
+};
+}  // namespace hat
+
 struct hat_plan {
     // geometry the plan was made for
     int32_t dtype, num_pages, num_heads, head_dim, max_pages, num_requests, total_rows;
@@ -76,6 +86,7 @@ struct hat_plan {
     std::vector<hat::MergeRow> merge_rows;
     int64_t part_rows;          // partial rows in the workspace
     hat_plan_info info;
+    hat::Timing* timing;        // null unless hat_plan_enable_timing was called
     void* dev_blob;             // one allocation holding every device array
     hat::DevicePlan dev;
 };
