@@ -223,6 +223,51 @@ int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num
  */
 int hat_last_device_status(const hat_plan* plan, void* stream, int* out);
 
+/*
+ * Streaming attention for callers that must not allocate.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)
+ *
+ * Who needs it: a serving loop that runs under CUDA-graph capture or inside a
+ * framework that has handed the whole device heap to its own allocator cannot
+ * call cudaMalloc, so it can neither create a hat_plan nor obtain the workspace
+ * hat_chunk_attention wants for its split-KV partial results.  This entry point
+ * computes the same out/lse as hat_chunk_attention for short chunks
+ * (chunk_len <= max_chunk_len <= 16, i.e. draft verification and decode) and
+ * calls no cudaMalloc / cudaFree or any allocating routine.  Its partial
+ * results go to a fixed array of HAT_STATIC_SCRATCH_BYTES that is part of the
+ * library's device code: every GPU that loads the library holds that much
+ * memory until the process exits.
+ *
+ * Differences from hat_chunk_attention:
+ *   - cu_chunk, prefix_len, chunk_len, block_table are DEVICE arrays (same
+ *     shapes and meaning as in hat_batch_desc); the host cannot inspect them,
+ *     so they are not validated: page ids are clamped into the pool and rows at
+ *     or beyond max_chunk_len are not computed.
+ *   - No append: the chunk's K/V must already be in the cache.
+ *   - Every request is cut into HAT_STATIC_SPLITS key ranges of equal length.
+ *   - Limit: num_requests * HAT_STATIC_SPLITS * max_chunk_len * heads * (head_dim+1) * 4 bytes
+ *     (rounded up to 256) must fit in HAT_STATIC_SCRATCH_BYTES, and
+ *     num_requests * HAT_STATIC_SPLITS <= 65535; otherwise HAT_ERR_TOO_LARGE
+ *     and nothing is launched.
+ *   - The first call on each device looks up the device address of the scratch
+ *     array (cudaGetSymbolAddress, with that device current); make that first
+ *     call outside any stream capture.
+ *   - All calls on one GPU share the scratch array, which keeps the previous
+ *     call's partial results; each call overwrites every slot it later reads,
+ *     so nothing has to be cleared, but two calls that overlap in time on the
+ *     same GPU (different streams) race on it.  Serialise them.
+ * Errors: INVALID_ARG, UNSUPPORTED, TOO_LARGE, CUDA (the cudaError_t is then
+ * available from cudaPeekAtLastError, not from hat_last_cuda_error).
+ */
+#define HAT_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+#define HAT_STATIC_SPLITS 8
+int hat_verify_attention_static(const hat_cache_desc* cache, int num_requests, int num_q_heads,
+                                int max_chunk_len, int max_pages,
+                                const int32_t* cu_chunk, const int32_t* prefix_len,      /* device */
+                                const int32_t* chunk_len, const int32_t* block_table,    /* device */
+                                const void* q, float* out, float* lse,                   /* device */
+                                float sm_scale, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

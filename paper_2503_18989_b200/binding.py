@@ -34,7 +34,10 @@ EXPORTS = [
     "hat_plan_create", "hat_plan_get_info", "hat_plan_workspace_bytes", "hat_plan_destroy",
     "hat_kv_append", "hat_chunk_attention", "hat_plan_staging_bytes", "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
+    "hat_verify_attention_static",
 ]
+HAT_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+HAT_STATIC_SPLITS = 8
 HAT_TIMING_SLOTS = 4
 
 
@@ -115,6 +118,9 @@ def lib() -> C.CDLL:
         L.hat_plan_enable_timing.argtypes = [vp, i32]
         L.hat_plan_read_timing.restype = i32
         L.hat_plan_read_timing.argtypes = [vp, vp, i32, C.POINTER(i32)]
+        L.hat_verify_attention_static.restype = i32
+        L.hat_verify_attention_static.argtypes = [C.POINTER(hat_cache_desc), i32, i32, i32, i32, vp, vp, vp, vp,
+                                                  vp, vp, vp, C.c_float, vp]
         _lib = L
     return _lib
 
@@ -255,3 +261,13 @@ def hat_plan_read_timing(plan, capacity_calls: int) -> np.ndarray:
     n = C.c_int()
     _check(lib().hat_plan_read_timing(_h(plan), _ptr(ms), int(capacity_calls), C.byref(n)), "hat_plan_read_timing")
     return ms[: n.value]
+
+
+def hat_verify_attention_static(cache: hat_cache_desc, num_requests: int, num_q_heads: int, max_chunk_len: int,
+                                max_pages: int, cu_chunk, prefix_len, chunk_len, block_table, q, out, lse,
+                                sm_scale: float = 0.0, stream: int = 0) -> None:
+    """Allocation-free streaming attention; the four descriptor arrays are DEVICE int32 tensors."""
+    _check(lib().hat_verify_attention_static(C.byref(cache), int(num_requests), int(num_q_heads),
+                                             int(max_chunk_len), int(max_pages), _ptr(cu_chunk), _ptr(prefix_len),
+                                             _ptr(chunk_len), _ptr(block_table), _ptr(q), _ptr(out), _ptr(lse),
+                                             float(sm_scale), stream or None), "hat_verify_attention_static")
