@@ -1,0 +1,520 @@
+// Prefill-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+// One CTA = 128 query rows of one request x one head x one key range.  Roles:
+//   warp 0      TMA producer: Q tile once, then K and V tiles of 128 keys (8 pages x 2 halves of 64 columns,
+//               128-byte swizzle) into two-stage rings, completion on mbarriers
+//   warp 1      one thread issues tcgen05.mma: S = Q K^T into one of two TMEM buffers, then O += P V with P read
+//               from TMEM; tcgen05.commit signals the consumers and frees the ring slots.  Owns the TMEM allocation
+//   warps 2-5   128 threads, thread = query row = TMEM lane: tcgen05.ld of S, scale/mask/online softmax in
+//               registers (running maximum only moved when it grows by more than 2^8, so O is rarely rescaled),
+//               P written back to TMEM as the 16-bit A operand, final O / l and log-sum-exp to global memory
+// TMEM columns: S0 [0,128) S1 [128,256) O [256,384).  P(j) overwrites the S buffer it was computed from (16-bit pairs in
+// columns [0,64), the bf16 rounding remainder in [64,128)); the next S into that buffer is issued after P V(j) by the
+// same thread, and tcgen05 executes one thread's MMAs in issue order, so no extra barrier guards the reuse.
+// Every wait is bounded (about a second); a wait that gives up sets the plan's status word, raises a CTA-wide abort
+// flag that all other waits observe, and the CTA still frees its TMEM and exits normally.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "hat_internal.h"
+
+namespace hat {
+namespace {
+
+constexpr int kRows = 128;      // query rows per CTA (MMA M)
+constexpr int kKeys = 128;      // keys per tile (MMA N of S, K extent of PV)
+constexpr int kD = 128;         // head_dim
+constexpr int kStages = 2;
+constexpr uint32_t kTileBytes = kKeys * kD * 2;          // 32 KiB: one K or V tile, or the Q tile
+constexpr uint32_t kSlabBytes = kKeys * 64 * 2;          // 16 KiB: 64 columns of 128 rows
+constexpr uint32_t kPageBoxBytes = 16 * 64 * 2;          // 2 KiB: one TMA box (16 tokens x 64 columns)
+constexpr float kRescaleThreshold = 8.0f;                // log2 units
+constexpr long long kWaitCycles = 2000000000LL;          // about a second at B200 clocks
+
+struct __align__(8) Barriers {
+    uint64_t q_full;
+    uint64_t k_full[kStages], k_empty[kStages];
+    uint64_t v_full[kStages], v_empty[kStages];
+    uint64_t s_full[2];
+    uint64_t p_ready, o_done, drain;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (1 + 2 * kStages) + 256;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the wait gave up or another role already did.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* b, int32_t* status) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity)) {
+        if (b->abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            b->abort_flag = 1;
+            atomicExch(status, 1);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+
+#define HAT_R32(r, o) "=r"(r[o+0]), "=r"(r[o+1]), "=r"(r[o+2]), "=r"(r[o+3]), "=r"(r[o+4]), "=r"(r[o+5]), "=r"(r[o+6]), "=r"(r[o+7])
+#define HAT_W32(r, o) "r"(r[o+0]), "r"(r[o+1]), "r"(r[o+2]), "r"(r[o+3]), "r"(r[o+4]), "r"(r[o+5]), "r"(r[o+6]), "r"(r[o+7])
+// 32 consecutive 32-bit columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : HAT_R32(r, 0), HAT_R32(r, 8), HAT_R32(r, 16), HAT_R32(r, 24)
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+        ::"r"(taddr), HAT_W32(r, 0), HAT_W32(r, 8), HAT_W32(r, 16), HAT_W32(r, 24) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+        ::"r"(taddr), HAT_W32(r, 0), HAT_W32(r, 8) : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor for kind::f16: fp32 accumulate, 16-bit A/B of type `fmt` (0 = f16, 1 = bf16).
+__host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, uint32_t b_mn_major, uint32_t m, uint32_t n) {
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((m >> 4) << 24);
+}
+
+template <bool BF16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    if constexpr (BF16) {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    } else {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(192, 1)
+attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_constant__ CUtensorMap map_q,
+                const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment: the swizzle pattern and the matrix descriptors assume it
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* q_tile = smem;
+    unsigned char* k_ring = smem + kTileBytes;
+    unsigned char* v_ring = k_ring + kStages * kTileBytes;
+    Barriers* bars = reinterpret_cast<Barriers*>(v_ring + kStages * kTileBytes);
+
+    const WorkItem item = items[blockIdx.y];
+    const int h = blockIdx.x;
+    const int H = a.plan.num_heads;
+    const int r = item.req;
+    const int P = a.plan.prefix_len[r];
+    const int C = a.plan.chunk_len[r];
+    const int row_base = a.plan.cu_chunk[r];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = (item.kv_end - item.kv_begin + kKeys - 1) / kKeys;
+    int32_t* status = a.plan.status;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bars->q_full, 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
+            mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
+        }
+        for (int s = 0; s < 2; ++s) mbar_init(&bars->s_full[s], 1);
+        mbar_init(&bars->p_ready, 128);
+        mbar_init(&bars->o_done, 1);
+        mbar_init(&bars->drain, 1);
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;\n" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    const uint32_t tm_s[2] = {tmem, tmem + 128};
+    const uint32_t tm_o = tmem + 256;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        const int32_t* __restrict__ table = a.plan.block_table + (int64_t)r * a.plan.max_pages;
+        if (lane == 0) mbar_expect_tx(&bars->q_full, kTileBytes);
+        __syncwarp();
+        if (lane < 2) tma_load_3d(smem_u32(q_tile) + lane * kSlabBytes, &map_q, lane * 64, h, row_base + item.row0, &bars->q_full);
+        // lane l < 16 moves box (page l/2 of the tile, column half l%2)
+        const int pg = lane >> 1, half = lane & 1;
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int st = j % kStages;
+            const uint32_t ph = (j / kStages) & 1;
+            const int kb = item.kv_begin + j * kKeys;
+            const int npages = (min(item.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
+            int page = 0;
+            if (lane < 16 && pg < npages) page = __ldg(table + kb / kPageSize + pg);
+            // K tile
+            if (j >= kStages) ok = mbar_wait(&bars->k_empty[st], ph ^ 1, bars, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) mbar_expect_tx(&bars->k_full[st], npages * 2 * kPageBoxBytes);
+            __syncwarp();
+            if (lane < 16 && pg < npages)
+                tma_load_4d(smem_u32(k_ring) + st * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0, h,
+                            page, &bars->k_full[st]);
+            // V tile
+            if (j >= kStages) ok = mbar_wait(&bars->v_empty[st], ph ^ 1, bars, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) mbar_expect_tx(&bars->v_full[st], npages * 2 * kPageBoxBytes);
+            __syncwarp();
+            if (lane < 16 && pg < npages)
+                tma_load_4d(smem_u32(v_ring) + st * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0, h,
+                            page, &bars->v_full[st]);
+        }
+        if (!ok) {
+            // give copies already in flight a bounded chance to land before the CTA's shared memory is released
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000) { }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t fmt = BF16 ? 1u : 0u;
+            constexpr uint32_t idesc_s = make_idesc(fmt, 0, kRows, kKeys);   // Q (K-major) x K (K-major)
+            constexpr uint32_t idesc_o = make_idesc(fmt, 1, kRows, kD);      // P (TMEM)    x V (MN-major)
+            const uint32_t q_addr = smem_u32(q_tile);
+            bool ok = mbar_wait(&bars->q_full, 0, bars, status);
+            auto issue_s = [&](int j) {
+                const int st = j % kStages;
+                const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kD / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
+                    mma_ss(tm_s[j & 1], smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                }
+                tc_commit(&bars->k_empty[st]);
+                tc_commit(&bars->s_full[j & 1]);
+            };
+            if (ok) ok = mbar_wait(&bars->k_full[0], 0, bars, status);
+            if (ok) issue_s(0);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % kStages;
+                if (j + 1 < n_tiles) {
+                    const int jn = j + 1;
+                    // S buffer jn&1 held S(jn-2) and then P(jn-2): P V(jn-2) was issued by this thread in the
+                    // previous iteration, after the softmax threads had read S(jn-2), so the buffer is free
+                    ok = mbar_wait(&bars->k_full[jn % kStages], (jn / kStages) & 1, bars, status);
+                    if (!ok) break;
+                    issue_s(jn);
+                }
+                ok = mbar_wait(&bars->v_full[st], (j / kStages) & 1, bars, status);
+                if (ok) ok = mbar_wait(&bars->p_ready, j & 1, bars, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < kKeys / 16; ++ks) {
+                    // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
+                    const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
+                    mma_ts(tm_o, tm_s[j & 1] + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));
+                    if constexpr (BF16) mma_ts(tm_o, tm_s[j & 1] + 64 + ks * 8, vdesc, idesc_o, true);
+                }
+                tc_commit(&bars->v_empty[st]);
+                tc_commit(&bars->o_done);
+            }
+            if (!ok) {
+                // gave up: let the MMAs already issued finish (bounded) before TMEM is released
+                tc_commit(&bars->drain);
+                const long long t0 = clock64();
+                while (!mbar_try(&bars->drain, 0) && clock64() - t0 < kWaitCycles) { }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ softmax / correction / epilogue
+        const int quarter = warp & 3;                       // TMEM lanes this warp may touch
+        const int t = quarter * 32 + lane;                  // query row inside the tile = TMEM lane
+        const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
+        const int i_row = item.row0 + t;                    // row inside the chunk
+        const int last_key = min(P + i_row, item.kv_end - 1);
+        float m_used = -INFINITY, l = 0.f;                  // scaled by scale_log2
+        const float sc = a.scale_log2;
+        bool ok = true;
+        for (int j = 0; j < n_tiles; ++j) {
+            const int b = j & 1;
+            const int kb = item.kv_begin + j * kKeys;
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[b], (j >> 1) & 1, bars, status));
+            if (!ok) break;
+            tc_fence_after();
+            float s[kKeys];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tm_s[b] + lane_sel + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
+            tmem_ld_wait();
+
+            // raw maximum (the scale is positive, so it commutes with max)
+            float mx = -INFINITY;
+            const int lim = last_key - kb;                  // keys 0..lim of this tile are visible to this row
+            if (lim < kKeys - 1) {
+#pragma unroll
+                for (int k = 0; k < kKeys; ++k) {
+                    s[k] = (k <= lim) ? s[k] : -INFINITY;
+                    mx = fmaxf(mx, s[k]);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < kKeys; ++k) mx = fmaxf(mx, s[k]);
+            }
+            mx *= sc;
+            // move the reference maximum only when it grew by more than the threshold
+            float alpha = 1.f;
+            bool rescale = false;
+            if (mx > m_used + kRescaleThreshold) {
+                alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
+                rescale = (m_used != -INFINITY);
+                m_used = mx;
+            }
+            const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t p[16];
+                uint32_t pl[16];
+#pragma unroll
+                for (int k = 0; k < 32; k += 2) {
+                    const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
+                    const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
+                    sum += e0 + e1;
+                    p[k / 2] = pack2<BF16>(e0, e1);
+                    if constexpr (BF16) {
+                        const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
+                        const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
+                        pl[k / 2] = pack2<BF16>(r0, r1);
+                    }
+                }
+                tmem_st16(tm_s[b] + lane_sel + c * 16, p);
+                if constexpr (BF16) tmem_st16(tm_s[b] + lane_sel + 64 + c * 16, pl);
+            }
+            l = l * alpha + sum;
+
+            // O may only be rescaled once the previous P V product has finished; waiting here every tile (it has
+            // long completed by now) also keeps this thread's view of the barrier phase in step
+            if (j > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done, (j - 1) & 1, bars, status));
+                if (!ok) break;
+                tc_fence_after();
+            }
+            if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tm_o + lane_sel + c * 32, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                    tmem_st32(tm_o + lane_sel + c * 32, o);
+                }
+            }
+            tmem_st_wait();
+            // last tile of a range that ends inside it: V rows past the range were not loaded (or hold
+            // stale slots); zero them so that 0 * garbage cannot produce NaN
+            if (kb + kKeys > item.kv_end) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[j % kStages], (j / kStages) & 1, bars, status));
+                if (!ok) break;
+                unsigned char* vt = v_ring + (j % kStages) * kTileBytes;
+                const int first = item.kv_end - kb;
+                for (int idx = (int)threadIdx.x - 64; idx < (kKeys - first) * 16; idx += 128) {
+                    const int row = first + idx / 16, part = idx % 16;      // 16 vectors of 16 bytes per 256-byte row
+                    *reinterpret_cast<uint4*>(vt + (part >> 3) * kSlabBytes + row * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
+                }
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+            }
+            tc_fence_before();
+            mbar_arrive(&bars->p_ready);
+        }
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done, (n_tiles - 1) & 1, bars, status));
+        if (ok) {
+            tc_fence_after();
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            const bool valid = i_row < C;
+            float* obase; float* lbase; int64_t orow;
+            if (item.part < 0) { obase = a.out; lbase = a.lse; orow = row_base + i_row; }
+            else { obase = a.part_out; lbase = a.part_lse; orow = item.part + t; }
+            float* dst = obase + (orow * H + h) * kD;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tm_o + lane_sel + c * 32, o);
+                tmem_ld_wait();
+                if (valid) {
+#pragma unroll
+                    for (int k = 0; k < 32; k += 4)
+                        *reinterpret_cast<float4*>(dst + c * 32 + k) =
+                            make_float4(__uint_as_float(o[k]) * inv, __uint_as_float(o[k + 1]) * inv,
+                                        __uint_as_float(o[k + 2]) * inv, __uint_as_float(o[k + 3]) * inv);
+                }
+            }
+            if (valid) lbase[orow * H + h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+bool encode_pool_map(CUtensorMap* map, bool bf16, const void* pool, int num_pages, int H, int64_t stride_page,
+                     int64_t stride_token, int64_t stride_head) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kPageSize, (cuuint64_t)H, (cuuint64_t)num_pages};
+    const cuuint64_t strides[3] = {(cuuint64_t)stride_token * 2, (cuuint64_t)stride_head * 2, (cuuint64_t)stride_page * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(pool),
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool encode_q_map(CUtensorMap* map, bool bf16, const void* q, int T, int H) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)T};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)H * kD * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kRows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(q), dims,
+              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
+                          int64_t stride_head) {
+    if (head_dim != kD || num_pages <= 0) return false;
+    CUtensorMap m;
+    // the encoder checks alignment and ranges only; any 16-byte aligned address will do for the probe
+    return encode_pool_map(&m, dtype == HAT_DTYPE_BF16, reinterpret_cast<const void*>(uintptr_t(1) << 30), num_pages, H,
+                           stride_page, stride_token, stride_head);
+}
+
+cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
+    const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
+    CUtensorMap mq, mk, mv;
+    if (!encode_q_map(&mq, bf16, args.q, plan->total_rows, plan->num_heads) ||
+        !encode_pool_map(&mk, bf16, args.cache.k_pool, plan->num_pages, plan->num_heads, args.cache.stride_page,
+                         args.cache.stride_token, args.cache.stride_head) ||
+        !encode_pool_map(&mv, bf16, args.cache.v_pool, plan->num_pages, plan->num_heads, args.cache.stride_page,
+                         args.cache.stride_token, args.cache.stride_head))
+        return cudaErrorInvalidValue;
+    const dim3 grid(plan->num_heads, (unsigned)plan->prefill_items.size());
+    cudaError_t e;
+    if (bf16) {
+        e = cudaFuncSetAttribute(attn_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attn_tc5_kernel<true><<<grid, 192, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
+    } else {
+        e = cudaFuncSetAttribute(attn_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attn_tc5_kernel<false><<<grid, 192, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace hat

@@ -73,15 +73,17 @@ static int split_len_for(int kv_end, int wanted, int granule) {
     return std::max(wanted, least);
 }
 
-static void schedule(hat_plan* p, int num_sms) {
+static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     const int H = p->num_heads;
     const int R = p->num_requests;
     hat_plan_info& info = p->info;
 
     const int verify_max_rows = 16;
-    const int tile_rows = 64;                     // mma.sync tile kernel: 4 warps x 16 rows
+    // tile kernel: tcgen05 with 128-row tiles and 128-key steps, or mma.sync with 4 warps x 16 rows and 64-key steps
+    const int tile_rows = use_tc5 ? 128 : 64;
+    const int key_granule = use_tc5 ? 128 : 64;
     info.prefill_tile_rows = tile_rows;
-    info.prefill_kernel = 0;
+    info.prefill_kernel = use_tc5 ? 1 : 0;
 
     // ---- streaming (verify-class) requests: fixed-length key ranges, shortened until the SMs are covered
     int64_t verify_tokens = 0;
@@ -120,10 +122,10 @@ static void schedule(hat_plan* p, int num_sms) {
         if (tiles > 0 && tiles * H < want_ctas) {
             // aim for want_ctas pieces of equal length, not shorter than 256 keys
             const int pieces = ceil_div((int)want_ctas, H);
-            psplit = std::max(256, round_up((int)((tile_keys + pieces - 1) / pieces), 64));
+            psplit = std::max(256, round_up((int)((tile_keys + pieces - 1) / pieces), key_granule));
         }
     }
-    if (psplit > 0) psplit = round_up(psplit, 64);
+    if (psplit > 0) psplit = round_up(psplit, key_granule);
     info.prefill_split_len = psplit;
 
     for (int r = 0; r < R; ++r) {
@@ -136,7 +138,7 @@ static void schedule(hat_plan* p, int num_sms) {
             for (int row0 = 0; row0 < C; row0 += tile_rows) {
                 int rows_valid = std::min(tile_rows, C - row0);
                 int kv_end = P + row0 + rows_valid;
-                int sl = psplit > 0 ? split_len_for(kv_end, psplit, 64) : 0;
+                int sl = psplit > 0 ? split_len_for(kv_end, psplit, key_granule) : 0;
                 emit_tile(p, p->prefill_items, r, row0, rows_valid, kv_end, sl);
             }
         }
@@ -325,7 +327,14 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) { delete p; return cuda_fail(e); }
     }
-    schedule(p, num_sms);
+    // the tcgen05 tile kernel needs head_dim 128 and a pool layout a TMA descriptor can express
+    bool use_tc5 = p->head_dim == 128;
+    if (const char* k = std::getenv("HAT_PREFILL_KERNEL"))
+        if (std::strcmp(k, "mma") == 0) use_tc5 = false;
+    if (use_tc5 && !p->host_only)
+        use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
+                                       cache->stride_token, cache->stride_head);
+    schedule(p, num_sms, use_tc5);
 
     if (!p->host_only) {
         st = upload(p);
@@ -422,7 +431,8 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
     a.scale_log2 = sm_scale * 1.4426950408889634f;
 
     if (!plan->prefill_items.empty()) {
-        e = launch_attn_mma(plan, a, /*verify_class=*/false, s);
+        e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
+                                           : launch_attn_mma(plan, a, /*verify_class=*/false, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ran(1);
     }

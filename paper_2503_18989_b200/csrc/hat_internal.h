@@ -97,5 +97,9 @@ cudaError_t launch_kv_append(const hat_plan* plan, const CacheView& cache, void*
                              const void* k_new, const void* v_new, cudaStream_t stream);
 cudaError_t launch_attn_mma(const hat_plan* plan, const AttnArgs& args, bool verify_class, cudaStream_t stream);
 cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+// tcgen05 tile kernel (head_dim 128): whether a TMA descriptor can be built for this pool layout, and the launcher
+bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
+                          int64_t stride_head);
+cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
 void count_launch(int n = 1);
 }  // namespace hat
