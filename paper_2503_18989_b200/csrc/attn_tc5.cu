@@ -1,16 +1,18 @@
 // Prefill-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
 //
-// One CTA = 128 query rows of one request x one head x one key range.  Roles:
+// One CTA = up to 256 query rows (two 128-row query tiles) of one request x one head x one key range; both query
+// tiles use the same K/V tiles in shared memory, and while one tile's softmax runs the tensor pipe works for the
+// other.  Roles:
 //   warp 0      TMA producer: Q tile once, then K and V tiles of 128 keys (8 pages x 2 halves of 64 columns,
 //               128-byte swizzle) into two-stage rings, completion on mbarriers
-//   warp 1      one thread issues tcgen05.mma: S = Q K^T into one of two TMEM buffers, then O += P V with P read
+//   warp 1      one thread issues tcgen05.mma: S_t = Q_t K^T for query tile t, then O_t += P_t V with P read
 //               from TMEM; tcgen05.commit signals the consumers and frees the ring slots.  Owns the TMEM allocation
-//   warps 2-5   128 threads, thread = query row = TMEM lane: tcgen05.ld of S, scale/mask/online softmax in
+//   warps 2-5, 6-9   one warpgroup per query tile, thread = query row = TMEM lane: tcgen05.ld of S, scale/mask/online softmax in
 //               registers (running maximum only moved when it grows by more than 2^8, so O is rarely rescaled),
 //               P written back to TMEM as the 16-bit A operand, final O / l and log-sum-exp to global memory
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384).  P(j) overwrites the S buffer it was computed from (16-bit pairs in
-// columns [0,64), the bf16 rounding remainder in [64,128)); the next S into that buffer is issued after P V(j) by the
-// same thread, and tcgen05 executes one thread's MMAs in issue order, so no extra barrier guards the reuse.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512).  P_t(j) overwrites S_t(j) in place (16-bit pairs in
+// columns [0,64), the bf16 rounding remainder in [64,128)); S_t(j+1) is issued after P_t V(j) by the same thread, and
+// tcgen05 executes one thread's MMAs in issue order, so no extra barrier guards the reuse.
 // Every wait is bounded (about a second); a wait that gives up sets the plan's status word, raises a CTA-wide abort
 // flag that all other waits observe, and the CTA still frees its TMEM and exits normally.
 #include <cuda.h>
@@ -36,12 +38,13 @@ struct __align__(8) Barriers {
     uint64_t q_full;
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t v_full[kStages], v_empty[kStages];
-    uint64_t s_full[2];
-    uint64_t p_ready, o_done, drain;
+    uint64_t s_full[2], p_ready[2], o_done[2];   // per query tile
+    uint64_t drain;
     uint32_t tmem_base;
     volatile int abort_flag;
 };
-constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (1 + 2 * kStages) + 256;
+constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + 2 * kStages) + 256;
+constexpr int kThreads = 320;   // producer warp, MMA warp, two softmax warpgroups
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -163,14 +166,14 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_constant__ CUtensorMap map_q,
                 const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle pattern and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* q_tile = smem;
-    unsigned char* k_ring = smem + kTileBytes;
+    unsigned char* q_tiles = smem;                               // 2 x 32 KiB
+    unsigned char* k_ring = smem + 2 * kTileBytes;
     unsigned char* v_ring = k_ring + kStages * kTileBytes;
     Barriers* bars = reinterpret_cast<Barriers*>(v_ring + kStages * kTileBytes);
 
@@ -182,7 +185,11 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
     const int C = a.plan.chunk_len[r];
     const int row_base = a.plan.cu_chunk[r];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = (item.kv_end - item.kv_begin + kKeys - 1) / kKeys;
+    // the item's rows form up to two 128-row query tiles; tile 0 does not see the keys past its own last row
+    const int nq = (C - item.row0 > kRows) ? 2 : 1;
+    const int n_all = (item.kv_end - item.kv_begin + kKeys - 1) / kKeys;
+    const int end0 = min(item.kv_end, P + item.row0 + kRows);
+    const int n_q0 = nq == 1 ? n_all : max(0, (end0 - item.kv_begin + kKeys - 1) / kKeys);
     int32_t* status = a.plan.status;
 
     if (threadIdx.x == 0) {
@@ -191,9 +198,11 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
             mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
         }
-        for (int s = 0; s < 2; ++s) mbar_init(&bars->s_full[s], 1);
-        mbar_init(&bars->p_ready, 128);
-        mbar_init(&bars->o_done, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->s_full[s], 1);
+            mbar_init(&bars->p_ready[s], 128);
+            mbar_init(&bars->o_done[s], 1);
+        }
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -207,26 +216,25 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
-    const uint32_t tm_s[2] = {tmem, tmem + 128};
-    const uint32_t tm_o = tmem + 256;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         const int32_t* __restrict__ table = a.plan.block_table + (int64_t)r * a.plan.max_pages;
-        if (lane == 0) mbar_expect_tx(&bars->q_full, kTileBytes);
+        if (lane == 0) mbar_expect_tx(&bars->q_full, nq * kTileBytes);
         __syncwarp();
-        if (lane < 2) tma_load_3d(smem_u32(q_tile) + lane * kSlabBytes, &map_q, lane * 64, h, row_base + item.row0, &bars->q_full);
+        if (lane < 2 * nq)      // lane = 2 * (query tile) + (column half)
+            tma_load_3d(smem_u32(q_tiles) + (lane >> 1) * kTileBytes + (lane & 1) * kSlabBytes, &map_q, (lane & 1) * 64, h,
+                        row_base + item.row0 + (lane >> 1) * kRows, &bars->q_full);
         // lane l < 16 moves box (page l/2 of the tile, column half l%2)
         const int pg = lane >> 1, half = lane & 1;
         bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
+        for (int j = 0; j < n_all; ++j) {
             const int st = j % kStages;
             const uint32_t ph = (j / kStages) & 1;
             const int kb = item.kv_begin + j * kKeys;
             const int npages = (min(item.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
             int page = 0;
             if (lane < 16 && pg < npages) page = __ldg(table + kb / kPageSize + pg);
-            // K tile
             if (j >= kStages) ok = mbar_wait(&bars->k_empty[st], ph ^ 1, bars, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -235,7 +243,6 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             if (lane < 16 && pg < npages)
                 tma_load_4d(smem_u32(k_ring) + st * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0, h,
                             page, &bars->k_full[st]);
-            // V tile
             if (j >= kStages) ok = mbar_wait(&bars->v_empty[st], ph ^ 1, bars, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -256,46 +263,62 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             constexpr uint32_t fmt = BF16 ? 1u : 0u;
             constexpr uint32_t idesc_s = make_idesc(fmt, 0, kRows, kKeys);   // Q (K-major) x K (K-major)
             constexpr uint32_t idesc_o = make_idesc(fmt, 1, kRows, kD);      // P (TMEM)    x V (MN-major)
-            const uint32_t q_addr = smem_u32(q_tile);
             bool ok = mbar_wait(&bars->q_full, 0, bars, status);
-            auto issue_s = [&](int j) {
+            int k_ready = -1, v_ready = -1;                                  // last K / V tile known to have landed
+            // S_qt(j) = Q_qt K(j)^T into TMEM columns [128 qt, 128 qt + 128)
+            auto issue_s = [&](int qt, int j) {
                 const int st = j % kStages;
+                if (k_ready < j) {
+                    ok = mbar_wait(&bars->k_full[st], (j / kStages) & 1, bars, status);
+                    k_ready = j;
+                    if (!ok) return;
+                }
+                const uint32_t q_addr = smem_u32(q_tiles) + qt * kTileBytes;
                 const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < kD / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
-                    mma_ss(tm_s[j & 1], smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                    mma_ss(tmem + qt * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
                 }
-                tc_commit(&bars->k_empty[st]);
-                tc_commit(&bars->s_full[j & 1]);
+                tc_commit(&bars->s_full[qt]);
+                if (qt == nq - 1) tc_commit(&bars->k_empty[st]);             // the last reader of this K tile
             };
-            if (ok) ok = mbar_wait(&bars->k_full[0], 0, bars, status);
-            if (ok) issue_s(0);
-            for (int j = 0; j < n_tiles && ok; ++j) {
+            // O_qt (+)= P_qt(j) V(j); P sits in the columns S_qt(j) was computed in
+            auto issue_pv = [&](int qt, int j) {
                 const int st = j % kStages;
-                if (j + 1 < n_tiles) {
-                    const int jn = j + 1;
-                    // S buffer jn&1 held S(jn-2) and then P(jn-2): P V(jn-2) was issued by this thread in the
-                    // previous iteration, after the softmax threads had read S(jn-2), so the buffer is free
-                    ok = mbar_wait(&bars->k_full[jn % kStages], (jn / kStages) & 1, bars, status);
-                    if (!ok) break;
-                    issue_s(jn);
+                if (v_ready < j) {
+                    ok = mbar_wait(&bars->v_full[st], (j / kStages) & 1, bars, status);
+                    v_ready = j;
+                    if (!ok) return;
                 }
-                ok = mbar_wait(&bars->v_full[st], (j / kStages) & 1, bars, status);
-                if (ok) ok = mbar_wait(&bars->p_ready, j & 1, bars, status);
-                if (!ok) break;
+                ok = mbar_wait(&bars->p_ready[qt], j & 1, bars, status);
+                if (!ok) return;
                 tc_fence_after();
                 const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
+                const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
 #pragma unroll
                 for (int ks = 0; ks < kKeys / 16; ++ks) {
                     // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
                     const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
-                    mma_ts(tm_o, tm_s[j & 1] + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));
-                    if constexpr (BF16) mma_ts(tm_o, tm_s[j & 1] + 64 + ks * 8, vdesc, idesc_o, true);
+                    mma_ts(to, tp + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));
+                    if constexpr (BF16) mma_ts(to, tp + 64 + ks * 8, vdesc, idesc_o, true);
                 }
-                tc_commit(&bars->v_empty[st]);
-                tc_commit(&bars->o_done);
+                tc_commit(&bars->o_done[qt]);
+                if (qt == nq - 1) tc_commit(&bars->v_empty[st]);
+            };
+            if (ok && n_q0 > 0) issue_s(0, 0);
+            if (ok && nq == 2) issue_s(1, 0);
+            for (int j = 0; j < n_all && ok; ++j) {
+                // tile 0's P V(j), then at once its next S: the tensor pipe works on them while tile 1's softmax runs
+                if (j < n_q0) {
+                    issue_pv(0, j);
+                    if (ok && j + 1 < n_q0) issue_s(0, j + 1);
+                }
+                if (ok && nq == 2) {
+                    issue_pv(1, j);
+                    if (ok && j + 1 < n_all) issue_s(1, j + 1);
+                }
             }
             if (!ok) {
                 // gave up: let the MMAs already issued finish (bounded) before TMEM is released
@@ -307,128 +330,137 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax / correction / epilogue
+        const int qt = (warp - 2) >> 2;                     // query tile of this warpgroup
         const int quarter = warp & 3;                       // TMEM lanes this warp may touch
         const int t = quarter * 32 + lane;                  // query row inside the tile = TMEM lane
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-        const int i_row = item.row0 + t;                    // row inside the chunk
+        const uint32_t tm_s = tmem + qt * 128 + lane_sel, tm_o = tmem + 256 + qt * 128 + lane_sel;
+        const int n_mine = (qt == 0) ? n_q0 : n_all;
+        const int i_row = item.row0 + qt * kRows + t;       // row inside the chunk
         const int last_key = min(P + i_row, item.kv_end - 1);
-        float m_used = -INFINITY, l = 0.f;                  // scaled by scale_log2
+        const int wg_tid = (int)threadIdx.x - 64 - qt * 128;
+        float m_used = -INFINITY, l = 0.f;                  // in units of scale_log2
         const float sc = a.scale_log2;
         bool ok = true;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int b = j & 1;
-            const int kb = item.kv_begin + j * kKeys;
-            ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[b], (j >> 1) & 1, bars, status));
-            if (!ok) break;
-            tc_fence_after();
-            float s[kKeys];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tm_s[b] + lane_sel + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
-            tmem_ld_wait();
-
-            // raw maximum (the scale is positive, so it commutes with max)
-            float mx = -INFINITY;
-            const int lim = last_key - kb;                  // keys 0..lim of this tile are visible to this row
-            if (lim < kKeys - 1) {
-#pragma unroll
-                for (int k = 0; k < kKeys; ++k) {
-                    s[k] = (k <= lim) ? s[k] : -INFINITY;
-                    mx = fmaxf(mx, s[k]);
-                }
-            } else {
-#pragma unroll
-                for (int k = 0; k < kKeys; ++k) mx = fmaxf(mx, s[k]);
-            }
-            mx *= sc;
-            // move the reference maximum only when it grew by more than the threshold
-            float alpha = 1.f;
-            bool rescale = false;
-            if (mx > m_used + kRescaleThreshold) {
-                alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
-                rescale = (m_used != -INFINITY);
-                m_used = mx;
-            }
-            const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
-            float sum = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t p[16];
-                uint32_t pl[16];
-#pragma unroll
-                for (int k = 0; k < 32; k += 2) {
-                    const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
-                    const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
-                    sum += e0 + e1;
-                    p[k / 2] = pack2<BF16>(e0, e1);
-                    if constexpr (BF16) {
-                        const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
-                        const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
-                        pl[k / 2] = pack2<BF16>(r0, r1);
-                    }
-                }
-                tmem_st16(tm_s[b] + lane_sel + c * 16, p);
-                if constexpr (BF16) tmem_st16(tm_s[b] + lane_sel + 64 + c * 16, pl);
-            }
-            l = l * alpha + sum;
-
-            // O may only be rescaled once the previous P V product has finished; waiting here every tile (it has
-            // long completed by now) also keeps this thread's view of the barrier phase in step
-            if (j > 0) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done, (j - 1) & 1, bars, status));
+        if (qt < nq) {
+            for (int j = 0; j < n_mine; ++j) {
+                const int kb = item.kv_begin + j * kKeys;
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[qt], j & 1, bars, status));
                 if (!ok) break;
                 tc_fence_after();
+                float s[kKeys];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
+                tmem_ld_wait();
+
+                // raw maximum (the scale is positive, so it commutes with max); four independent chains
+                const int lim = last_key - kb;              // keys 0..lim of this tile are visible to this row
+                if (lim < kKeys - 1) {
+#pragma unroll
+                    for (int k = 0; k < kKeys; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
+                }
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int k = 0; k < kKeys; k += 8) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], fmaxf(s[k + 2 * u], s[k + 2 * u + 1]));
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
+                // move the reference maximum only when it grew by more than the threshold
+                float alpha = 1.f;
+                bool rescale = false;
+                if (mx > m_used + kRescaleThreshold) {
+                    alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
+                    rescale = (m_used != -INFINITY);
+                    m_used = mx;
+                }
+                const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t p[16];
+                    uint32_t pl[16];
+#pragma unroll
+                    for (int k = 0; k < 32; k += 2) {
+                        const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
+                        const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
+                        sum4[(k >> 1) & 3] += e0 + e1;
+                        p[k / 2] = pack2<BF16>(e0, e1);
+                        if constexpr (BF16) {
+                            const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
+                            const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
+                            pl[k / 2] = pack2<BF16>(r0, r1);
+                        }
+                    }
+                    tmem_st16(tm_s + c * 16, p);
+                    if constexpr (BF16) tmem_st16(tm_s + 64 + c * 16, pl);
+                }
+                l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+
+                // O may only be rescaled once the previous P V product has finished; waiting here every tile (it
+                // has long completed by now) also keeps this thread's view of the barrier phase in step
+                if (j > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], (j - 1) & 1, bars, status));
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tm_o + c * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                        tmem_st32(tm_o + c * 32, o);
+                    }
+                }
+                tmem_st_wait();
+                // a range that ends inside this tile: V rows past the range were not loaded (or hold stale
+                // slots); zero them so that 0 * garbage cannot produce NaN (both warpgroups may do it: same zeros)
+                if (kb + kKeys > item.kv_end) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[j % kStages], (j / kStages) & 1, bars, status));
+                    if (!ok) break;
+                    unsigned char* vt = v_ring + (j % kStages) * kTileBytes;
+                    const int first = item.kv_end - kb;
+                    for (int idx = wg_tid; idx < (kKeys - first) * 16; idx += 128) {
+                        const int row = first + idx / 16, part = idx % 16;     // 16 vectors of 16 bytes per 256-byte row
+                        *reinterpret_cast<uint4*>(vt + (part >> 3) * kSlabBytes + row * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                }
+                tc_fence_before();
+                mbar_arrive(&bars->p_ready[qt]);
             }
-            if (__any_sync(0xffffffffu, rescale)) {
+            if (ok && n_mine > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], (n_mine - 1) & 1, bars, status));
+            if (ok) {
+                tc_fence_after();
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                const bool valid = i_row < C;
+                float* obase; float* lbase; int64_t orow;
+                if (item.part < 0) { obase = a.out; lbase = a.lse; orow = row_base + i_row; }
+                else { obase = a.part_out; lbase = a.part_lse; orow = item.part + qt * kRows + t; }
+                float* dst = obase + (orow * H + h) * kD;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
-                    tmem_ld32(tm_o + lane_sel + c * 32, o);
-                    tmem_ld_wait();
+                    if (n_mine > 0) {                       // uniform over the warpgroup
+                        tmem_ld32(tm_o + c * 32, o);
+                        tmem_ld_wait();
+                    } else {
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                    tmem_st32(tm_o + lane_sel + c * 32, o);
-                }
-            }
-            tmem_st_wait();
-            // last tile of a range that ends inside it: V rows past the range were not loaded (or hold
-            // stale slots); zero them so that 0 * garbage cannot produce NaN
-            if (kb + kKeys > item.kv_end) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[j % kStages], (j / kStages) & 1, bars, status));
-                if (!ok) break;
-                unsigned char* vt = v_ring + (j % kStages) * kTileBytes;
-                const int first = item.kv_end - kb;
-                for (int idx = (int)threadIdx.x - 64; idx < (kKeys - first) * 16; idx += 128) {
-                    const int row = first + idx / 16, part = idx % 16;      // 16 vectors of 16 bytes per 256-byte row
-                    *reinterpret_cast<uint4*>(vt + (part >> 3) * kSlabBytes + row * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
-                }
-                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-            }
-            tc_fence_before();
-            mbar_arrive(&bars->p_ready);
-        }
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done, (n_tiles - 1) & 1, bars, status));
-        if (ok) {
-            tc_fence_after();
-            const float inv = l > 0.f ? 1.f / l : 0.f;
-            const bool valid = i_row < C;
-            float* obase; float* lbase; int64_t orow;
-            if (item.part < 0) { obase = a.out; lbase = a.lse; orow = row_base + i_row; }
-            else { obase = a.part_out; lbase = a.part_lse; orow = item.part + t; }
-            float* dst = obase + (orow * H + h) * kD;
+                        for (int k = 0; k < 32; ++k) o[k] = 0u;
+                    }
+                    if (valid) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tm_o + lane_sel + c * 32, o);
-                tmem_ld_wait();
-                if (valid) {
-#pragma unroll
-                    for (int k = 0; k < 32; k += 4)
-                        *reinterpret_cast<float4*>(dst + c * 32 + k) =
-                            make_float4(__uint_as_float(o[k]) * inv, __uint_as_float(o[k + 1]) * inv,
-                                        __uint_as_float(o[k + 2]) * inv, __uint_as_float(o[k + 3]) * inv);
+                        for (int k = 0; k < 32; k += 4)
+                            *reinterpret_cast<float4*>(dst + c * 32 + k) =
+                                make_float4(__uint_as_float(o[k]) * inv, __uint_as_float(o[k + 1]) * inv,
+                                            __uint_as_float(o[k + 2]) * inv, __uint_as_float(o[k + 3]) * inv);
+                    }
                 }
+                if (valid) lbase[orow * H + h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
             }
-            if (valid) lbase[orow * H + h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
     }
 
@@ -507,11 +539,11 @@ cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStre
     if (bf16) {
         e = cudaFuncSetAttribute(attn_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_tc5_kernel<true><<<grid, 192, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
+        attn_tc5_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
     } else {
         e = cudaFuncSetAttribute(attn_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_tc5_kernel<false><<<grid, 192, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
+        attn_tc5_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
     }
     count_launch();
     return cudaGetLastError();

@@ -79,8 +79,8 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     hat_plan_info& info = p->info;
 
     const int verify_max_rows = 16;
-    // tile kernel: tcgen05 with 128-row tiles and 128-key steps, or mma.sync with 4 warps x 16 rows and 64-key steps
-    const int tile_rows = use_tc5 ? 128 : 64;
+    // tile kernel: tcgen05 with 256-row tiles (two 128-row MMA tiles) and 128-key steps, or mma.sync with 4 warps x 16 rows and 64-key steps
+    const int tile_rows = use_tc5 ? 256 : 64;
     const int key_granule = use_tc5 ? 128 : 64;
     info.prefill_tile_rows = tile_rows;
     info.prefill_kernel = use_tc5 ? 1 : 0;
