@@ -4,7 +4,7 @@
 // tiles use the same K/V tiles in shared memory, and while one tile's softmax runs the tensor pipe works for the
 // other.  Roles:
 //   warp 0      TMA producer: Q tile once, then K and V tiles of 128 keys (8 pages x 2 halves of 64 columns,
-//               128-byte swizzle) into two-stage rings, completion on mbarriers
+//               128-byte swizzle) into a two-slot K ring and a three-slot V ring, completion on mbarriers
 //   warp 1      one thread issues tcgen05.mma: S_t = Q_t K^T for query tile t, then O_t += P_t V with P read
 //               from TMEM; tcgen05.commit signals the consumers and frees the ring slots.  Owns the TMEM allocation
 //   warps 2-5, 6-9   one warpgroup per query tile, thread = query row = TMEM lane: tcgen05.ld of S, scale/mask/online softmax in
@@ -27,7 +27,8 @@ namespace {
 constexpr int kRows = 128;      // query rows per CTA (MMA M)
 constexpr int kKeys = 128;      // keys per tile (MMA N of S, K extent of PV)
 constexpr int kD = 128;         // head_dim
-constexpr int kStages = 2;
+constexpr int kStagesK = 2;     // ring slots for K tiles
+constexpr int kStagesV = 3;     // ring slots for V tiles (V is requested later in a step than K, so it gets the deeper ring)
 constexpr uint32_t kTileBytes = kKeys * kD * 2;          // 32 KiB: one K or V tile, or the Q tile
 constexpr uint32_t kSlabBytes = kKeys * 64 * 2;          // 16 KiB: 64 columns of 128 rows
 constexpr uint32_t kPageBoxBytes = 16 * 64 * 2;          // 2 KiB: one TMA box (16 tokens x 64 columns)
@@ -36,14 +37,14 @@ constexpr long long kWaitCycles = 2000000000LL;          // about a second at B2
 
 struct __align__(8) Barriers {
     uint64_t q_full;
-    uint64_t k_full[kStages], k_empty[kStages];
-    uint64_t v_full[kStages], v_empty[kStages];
+    uint64_t k_full[kStagesK], k_empty[kStagesK];
+    uint64_t v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], p_ready[2], o_done[2];   // per query tile
     uint64_t drain;
     uint32_t tmem_base;
     volatile int abort_flag;
 };
-constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + 2 * kStages) + 256;
+constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + kStagesK + kStagesV) + 256;
 constexpr int kThreads = 320;   // producer warp, MMA warp, two softmax warpgroups
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -174,8 +175,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* q_tiles = smem;                               // 2 x 32 KiB
     unsigned char* k_ring = smem + 2 * kTileBytes;
-    unsigned char* v_ring = k_ring + kStages * kTileBytes;
-    Barriers* bars = reinterpret_cast<Barriers*>(v_ring + kStages * kTileBytes);
+    unsigned char* v_ring = k_ring + kStagesK * kTileBytes;
+    Barriers* bars = reinterpret_cast<Barriers*>(v_ring + kStagesV * kTileBytes);
 
     const WorkItem item = items[blockIdx.y];
     const int h = blockIdx.x;
@@ -194,10 +195,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
 
     if (threadIdx.x == 0) {
         mbar_init(&bars->q_full, 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
-            mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
-        }
+        for (int s = 0; s < kStagesK; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+        for (int s = 0; s < kStagesV; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars->s_full[s], 1);
             mbar_init(&bars->p_ready[s], 128);
@@ -229,28 +228,27 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
         const int pg = lane >> 1, half = lane & 1;
         bool ok = true;
         for (int j = 0; j < n_all; ++j) {
-            const int st = j % kStages;
-            const uint32_t ph = (j / kStages) & 1;
+            const int sk = j % kStagesK, sv = j % kStagesV;
             const int kb = item.kv_begin + j * kKeys;
             const int npages = (min(item.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
             int page = 0;
             if (lane < 16 && pg < npages) page = __ldg(table + kb / kPageSize + pg);
-            if (j >= kStages) ok = mbar_wait(&bars->k_empty[st], ph ^ 1, bars, status);
+            if (j >= kStagesK) ok = mbar_wait(&bars->k_empty[sk], ((j / kStagesK) & 1) ^ 1, bars, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (lane == 0) mbar_expect_tx(&bars->k_full[st], npages * 2 * kPageBoxBytes);
+            if (lane == 0) mbar_expect_tx(&bars->k_full[sk], npages * 2 * kPageBoxBytes);
             __syncwarp();
             if (lane < 16 && pg < npages)
-                tma_load_4d(smem_u32(k_ring) + st * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0, h,
-                            page, &bars->k_full[st]);
-            if (j >= kStages) ok = mbar_wait(&bars->v_empty[st], ph ^ 1, bars, status);
+                tma_load_4d(smem_u32(k_ring) + sk * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0, h,
+                            page, &bars->k_full[sk]);
+            if (j >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((j / kStagesV) & 1) ^ 1, bars, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (lane == 0) mbar_expect_tx(&bars->v_full[st], npages * 2 * kPageBoxBytes);
+            if (lane == 0) mbar_expect_tx(&bars->v_full[sv], npages * 2 * kPageBoxBytes);
             __syncwarp();
             if (lane < 16 && pg < npages)
-                tma_load_4d(smem_u32(v_ring) + st * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0, h,
-                            page, &bars->v_full[st]);
+                tma_load_4d(smem_u32(v_ring) + sv * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0, h,
+                            page, &bars->v_full[sv]);
         }
         if (!ok) {
             // give copies already in flight a bounded chance to land before the CTA's shared memory is released
@@ -267,9 +265,9 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             int k_ready = -1, v_ready = -1;                                  // last K / V tile known to have landed
             // S_qt(j) = Q_qt K(j)^T into TMEM columns [128 qt, 128 qt + 128)
             auto issue_s = [&](int qt, int j) {
-                const int st = j % kStages;
+                const int st = j % kStagesK;
                 if (k_ready < j) {
-                    ok = mbar_wait(&bars->k_full[st], (j / kStages) & 1, bars, status);
+                    ok = mbar_wait(&bars->k_full[st], (j / kStagesK) & 1, bars, status);
                     k_ready = j;
                     if (!ok) return;
                 }
@@ -286,9 +284,9 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             };
             // O_qt (+)= P_qt(j) V(j); P sits in the columns S_qt(j) was computed in
             auto issue_pv = [&](int qt, int j) {
-                const int st = j % kStages;
+                const int st = j % kStagesV;
                 if (v_ready < j) {
-                    ok = mbar_wait(&bars->v_full[st], (j / kStages) & 1, bars, status);
+                    ok = mbar_wait(&bars->v_full[st], (j / kStagesV) & 1, bars, status);
                     v_ready = j;
                     if (!ok) return;
                 }
@@ -419,9 +417,9 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
                 // a range that ends inside this tile: V rows past the range were not loaded (or hold stale
                 // slots); zero them so that 0 * garbage cannot produce NaN (both warpgroups may do it: same zeros)
                 if (kb + kKeys > item.kv_end) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[j % kStages], (j / kStages) & 1, bars, status));
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[j % kStagesV], (j / kStagesV) & 1, bars, status));
                     if (!ok) break;
-                    unsigned char* vt = v_ring + (j % kStages) * kTileBytes;
+                    unsigned char* vt = v_ring + (j % kStagesV) * kTileBytes;
                     const int first = item.kv_end - kb;
                     for (int idx = wg_tid; idx < (kKeys - first) * 16; idx += 128) {
                         const int row = first + idx / 16, part = idx % 16;     // 16 vectors of 16 bytes per 256-byte row
