@@ -86,11 +86,9 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     info.prefill_kernel = use_tc5 ? 1 : 0;
 
     // ---- streaming (verify-class) requests: fixed-length key ranges, shortened until the SMs are covered
-    int64_t verify_tokens = 0;
     for (int r = 0; r < R; ++r) {
         int C = p->chunk_len[r];
         if (C >= 1 && C <= verify_max_rows) {
-            verify_tokens += p->prefix_len[r] + C;
             info.num_verify_requests++;
         } else if (C > verify_max_rows) {
             info.num_prefill_requests++;
@@ -98,9 +96,20 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     }
     int vsplit = env_int("HAT_VERIFY_SPLIT_LEN", 0);
     if (vsplit <= 0) {
-        vsplit = 512;
-        const int64_t want_ctas = (int64_t)num_sms * 8;
-        while (vsplit > 64 && (verify_tokens / vsplit + info.num_verify_requests) * H < want_ctas) vsplit /= 2;
+        // Long ranges stream best (a CTA's pipeline ramp and its cross-warp merge are paid once per range, and an
+        // unsplit request needs no merge pass): start unsplit and halve the range only while the grid would not
+        // give every SM about three rounds of two resident CTAs.
+        vsplit = 16384;
+        const int64_t want_ctas = (int64_t)num_sms * 6;
+        auto ctas_at = [&](int len) {
+            int64_t n = 0;
+            for (int r = 0; r < R; ++r) {
+                const int C = p->chunk_len[r];
+                if (C >= 1 && C <= verify_max_rows) n += ceil_div(p->prefix_len[r] + C, len);
+            }
+            return n * H;
+        };
+        while (vsplit > 256 && ctas_at(vsplit) < want_ctas) vsplit /= 2;
     }
     vsplit = std::max(kPageSize, round_up(vsplit, kPageSize));
     info.verify_split_len = vsplit;
