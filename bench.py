@@ -119,6 +119,30 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(inside)}
 
 
+# ----------------------------------------------------------------------------
+# replicas: the path has no inter-GPU exchange, so N ranks run N independent copies of the batch
+# ----------------------------------------------------------------------------
+def replica_seed(workload: str, rank: int) -> int:
+    """Seed of rank `rank`'s replica: the workload's own seed for rank 0, shifted by 1000 per rank."""
+    return W.SEED_BASE + list(W.WORKLOADS).index(workload) + 1 + 1000 * rank
+
+
+def max_over_ranks(values, world: int, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity when world == 1)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_value(flops_per_replica_step: int, world: int, ms_per_step: float) -> float:
+    """TFLOP/s of the whole job: every rank does the same amount of work in the (max-over-ranks) step time."""
+    return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
+
+
 def pick_oracle_sample(cache, st, rng, target_flops):
     """(request, row, head) units drawn uniformly over all (row, head) pairs until ~target_flops."""
     H, d = cache.num_heads, cache.head_dim
@@ -165,7 +189,7 @@ def run_reference(args, rank):
     units, fl = pick_oracle_sample(sc.cache, st, rng, 2e8)
     t0 = time.perf_counter(); O.attention_rows(sc.cache, sc.k_pool, sc.v_pool, st, units)
     rate = fl / max(time.perf_counter() - t0, 1e-6)
-    per_step = min(20.0, 150.0 / max(1, args.steps + args.warmup))
+    per_step = min(20.0, args.cpu_budget, 150.0 / max(1, args.steps + args.warmup))
     units, fl = pick_oracle_sample(sc.cache, st, rng, rate * per_step)
     for _ in range(args.warmup):
         O.attention_rows(sc.cache, sc.k_pool, sc.v_pool, st, units)
@@ -237,7 +261,7 @@ def main():
     peaks, peak_kind = load_peaks()
 
     # ---- inputs: one replica of the batch per rank (seeded; different values per rank)
-    sc = W.WORKLOADS[args.workload](seed=W.SEED_BASE + list(W.WORKLOADS).index(args.workload) + 1 + 1000 * rank)
+    sc = W.WORKLOADS[args.workload](seed=replica_seed(args.workload, rank))
     cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, device)
     steps = [runner.DeviceStep(cache, st) for st in sc.steps]
     works = [step_work(sc.cache, st) for st in sc.steps]
@@ -327,15 +351,12 @@ def main():
     d2h = sum(st.total_rows * sc.cache.num_heads * (sc.cache.head_dim + 1) * 4 for st in sc.steps)
 
     # ---- max over ranks
-    if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e_ms], world, device)
 
     if rank == 0:
         ms_per_step = elapsed_ms / K
-        value = world * total["flops"] / (ms_per_step * 1e-3) / 1e12
-        e2e_value = world * total["flops"] / (e2e_ms / Ke * 1e-3) / 1e12
+        value = whole_job_value(total["flops"], world, ms_per_step)
+        e2e_value = whole_job_value(total["flops"], world, e2e_ms / Ke)
 
         # per-kernel achieved throughput against its roofline
         avg = np.where(kernel_calls > 0, kernel_ms / np.maximum(kernel_calls, 1), 0.0)   # ms per launch
