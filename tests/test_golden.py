@@ -22,8 +22,8 @@ def test_oracle_reproduces_stored_values():
     rows = _load()
     assert len(rows) >= 15
     for s, i, h, out4, lse in rows:
-        assert np.array_equal(res[s][0][i, h, :4], out4)
-        assert res[s][1][i, h] == lse
+        assert np.allclose(res[s][0][i, h, :4], out4, rtol=0, atol=1e-12)    # libm may differ in the last bit
+        assert abs(res[s][1][i, h] - lse) <= 1e-12
 
 
 @pytest.mark.gpu
