@@ -143,6 +143,23 @@ def whole_job_value(flops_per_replica_step: int, world: int, ms_per_step: float)
     return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
 
 
+def lookup_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu capture of this kernel on this workload, or None when
+    there is none or the kernel source has changed since (profiles/traffic.json records a source hash)."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            table = json.load(f)["entries"]
+        for e in table:
+            if e["kernel"] == kernel and e["workload"] == workload:
+                with open(os.path.join(ROOT, e["source"]), "rb") as src:
+                    if hashlib.sha256(src.read()).hexdigest()[:16] == e["source_sha256_16"]:
+                        return int(e["traffic_bytes"])
+    except Exception:
+        pass
+    return None
+
+
 def pick_oracle_sample(cache, st, rng, target_flops):
     """(request, row, head) units drawn uniformly over all (row, head) pairs until ~target_flops."""
     H, d = cache.num_heads, cache.head_dim
@@ -382,7 +399,7 @@ def main():
                              "share": float(kernel_ms[i] / max(kernel_ms.sum(), 1e-9))}
         dominant = max(kernels, key=lambda n: kernels[n]["share"])
         roof = {k: kernels[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
-        roof.update({"kernel": dominant, "traffic": None, "peak_source": f"{peak_kind} "
+        roof.update({"kernel": dominant, "traffic": lookup_traffic(dominant, sc.name), "peak_source": f"{peak_kind} "
                      + ("bf16 sustained" if roof["bound"] == "tensor" else "HBM copy")})
         # the tile kernel against the memory roofline as well (short chunks are HBM-bound)
         if "tile_attention" in kernels:
