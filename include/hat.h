@@ -217,11 +217,26 @@ int hat_plan_enable_timing(hat_plan* plan, int max_calls);
 int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num_calls);
 
 /*
- * Read the device-side status word of a plan (synchronises `stream`).  *out is
- * HAT_OK, or HAT_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up
- * since the plan was created; results of such a call are undefined.
+ * Read and clear the device-side status word of a plan (synchronises
+ * `stream`).  *out is HAT_OK, or HAT_ERR_DEVICE_TIMEOUT if a bounded wait
+ * inside a kernel gave up since the word was last read; the results of the
+ * calls in between are then undefined, but the kernels have exited normally
+ * and the context stays usable.
  */
 int hat_last_device_status(const hat_plan* plan, void* stream, int* out);
+
+/*
+ * Failure detection of the tile kernel.  Every wait inside it (on a TMA
+ * transfer, on the tensor pipe, on another warp) is bounded by `cycles` SM
+ * clock cycles (0 selects the default of 2e9, about a second); a wait that
+ * runs out sets the status word above, tells the other warps of its CTA to
+ * stop, and the CTA releases its tensor memory and exits.
+ * withhold_next_call != 0 is a self test of that path: in the next
+ * hat_chunk_attention call on this plan every tile-kernel CTA skips one of
+ * its own transfers, so that a wait does run out within the bound; that call's
+ * out/lse are undefined.  Nothing faults or hangs.
+ */
+int hat_plan_set_wait_limit(hat_plan* plan, long long cycles, int withhold_next_call);
 
 /*
  * Streaming attention for callers that must not allocate.  (The paper has no

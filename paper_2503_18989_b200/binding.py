@@ -34,7 +34,7 @@ EXPORTS = [
     "hat_plan_create", "hat_plan_get_info", "hat_plan_workspace_bytes", "hat_plan_destroy",
     "hat_kv_append", "hat_chunk_attention", "hat_plan_staging_bytes", "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
-    "hat_verify_attention_static",
+    "hat_verify_attention_static", "hat_plan_set_wait_limit",
 ]
 HAT_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 HAT_STATIC_SPLITS = 8
@@ -118,6 +118,8 @@ def lib() -> C.CDLL:
         L.hat_plan_enable_timing.argtypes = [vp, i32]
         L.hat_plan_read_timing.restype = i32
         L.hat_plan_read_timing.argtypes = [vp, vp, i32, C.POINTER(i32)]
+        L.hat_plan_set_wait_limit.restype = i32
+        L.hat_plan_set_wait_limit.argtypes = [vp, C.c_longlong, i32]
         L.hat_verify_attention_static.restype = i32
         L.hat_verify_attention_static.argtypes = [C.POINTER(hat_cache_desc), i32, i32, i32, i32, vp, vp, vp, vp,
                                                   vp, vp, vp, C.c_float, vp]
@@ -271,3 +273,8 @@ def hat_verify_attention_static(cache: hat_cache_desc, num_requests: int, num_q_
                                              int(max_chunk_len), int(max_pages), _ptr(cu_chunk), _ptr(prefix_len),
                                              _ptr(chunk_len), _ptr(block_table), _ptr(q), _ptr(out), _ptr(lse),
                                              float(sm_scale), stream or None), "hat_verify_attention_static")
+
+
+def hat_plan_set_wait_limit(plan, cycles: int = 0, withhold_next_call: bool = False) -> None:
+    _check(lib().hat_plan_set_wait_limit(_h(plan), int(cycles), 1 if withhold_next_call else 0),
+           "hat_plan_set_wait_limit")

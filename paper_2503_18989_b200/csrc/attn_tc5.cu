@@ -13,7 +13,7 @@
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512).  P_t(j) overwrites S_t(j) in place (16-bit pairs in
 // columns [0,64), the bf16 rounding remainder in [64,128)); S_t(j+1) is issued after P_t V(j) by the same thread, and
 // tcgen05 executes one thread's MMAs in issue order, so no extra barrier guards the reuse.
-// Every wait is bounded (about a second); a wait that gives up sets the plan's status word, raises a CTA-wide abort
+// Every wait is bounded (about a second by default); a wait that gives up sets the plan's status word, raises a CTA-wide abort
 // flag that all other waits observe, and the CTA still frees its TMEM and exits normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -33,7 +33,6 @@ constexpr uint32_t kTileBytes = kKeys * kD * 2;          // 32 KiB: one K or V t
 constexpr uint32_t kSlabBytes = kKeys * 64 * 2;          // 16 KiB: 64 columns of 128 rows
 constexpr uint32_t kPageBoxBytes = 16 * 64 * 2;          // 2 KiB: one TMA box (16 tokens x 64 columns)
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
-constexpr long long kWaitCycles = 2000000000LL;          // about a second at B200 clocks
 
 struct __align__(8) Barriers {
     uint64_t q_full;
@@ -41,6 +40,7 @@ struct __align__(8) Barriers {
     uint64_t v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], p_ready[2], o_done[2];   // per query tile
     uint64_t drain;
+    long long wait_cycles;                       // bound of every wait below
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -73,7 +73,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barrie
     const long long t0 = clock64();
     while (!mbar_try(bar, parity)) {
         if (b->abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > b->wait_cycles) {
             b->abort_flag = 1;
             atomicExch(status, 1);
             return false;
@@ -204,6 +204,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
         }
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
+        bars->wait_cycles = a.wait_cycles;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
@@ -244,6 +245,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             if (j >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((j / kStagesV) & 1) ^ 1, bars, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            if (a.withhold && j == 0) continue;          // self test: this V tile never arrives, its consumers give up
             if (lane == 0) mbar_expect_tx(&bars->v_full[sv], npages * 2 * kPageBoxBytes);
             __syncwarp();
             if (lane < 16 && pg < npages)
@@ -322,7 +324,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
                 // gave up: let the MMAs already issued finish (bounded) before TMEM is released
                 tc_commit(&bars->drain);
                 const long long t0 = clock64();
-                while (!mbar_try(&bars->drain, 0) && clock64() - t0 < kWaitCycles) { }
+                while (!mbar_try(&bars->drain, 0) && clock64() - t0 < bars->wait_cycles) { }
             }
         }
         __syncwarp();

@@ -308,6 +308,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->part_rows = 0;
     p->dev_blob = nullptr;
     p->timing = nullptr;
+    p->wait_cycles = 2000000000LL;
+    p->withhold_next = 0;
     std::memset(&p->info, 0, sizeof p->info);
     std::memset(&p->dev, 0, sizeof p->dev);
     p->cu_chunk.assign(batch->cu_chunk, batch->cu_chunk + R + 1);
@@ -438,6 +440,9 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
     const size_t part_out_bytes = ((size_t)plan->part_rows * H * d * 4 + 255) / 256 * 256;
     a.part_lse = need ? reinterpret_cast<float*>(static_cast<char*>(workspace) + part_out_bytes) : nullptr;
     a.scale_log2 = sm_scale * 1.4426950408889634f;
+    a.wait_cycles = plan->wait_cycles;
+    a.withhold = plan->withhold_next;
+    const_cast<hat_plan*>(plan)->withhold_next = 0;
 
     if (!plan->prefill_items.empty()) {
         e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
@@ -555,9 +560,17 @@ int hat_last_device_status(const hat_plan* plan, void* stream, int* out) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int32_t word = 0;
     cudaError_t e = cudaMemcpyAsync(&word, plan->dev.status, sizeof word, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(plan->dev.status, 0, sizeof word, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
     *out = word == 0 ? HAT_OK : HAT_ERR_DEVICE_TIMEOUT;
+    return HAT_OK;
+}
+
+int hat_plan_set_wait_limit(hat_plan* plan, long long cycles, int withhold_next_call) {
+    if (!plan || cycles < 0) return HAT_ERR_INVALID_ARG;
+    plan->wait_cycles = cycles > 0 ? cycles : 2000000000LL;
+    plan->withhold_next = withhold_next_call ? 1 : 0;
     return HAT_OK;
 }
 

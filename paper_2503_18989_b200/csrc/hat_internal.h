@@ -62,6 +62,8 @@ struct AttnArgs {
     float*      part_out;     // [part_rows][H][d]
     float*      part_lse;     // [part_rows][H]
     float       scale_log2;   // sm_scale * log2(e)
+    long long   wait_cycles;  // bound of every device-side wait, in SM clock cycles
+    int         withhold;     // self test: the tile kernel's producer skips its first V tile so that a wait runs out
 };
 
 }  // namespace hat
@@ -87,6 +89,8 @@ struct hat_plan {
     int64_t part_rows;          // partial rows in the workspace
     hat_plan_info info;
     hat::Timing* timing;        // null unless hat_plan_enable_timing was called
+    long long wait_cycles;      // bound of device-side waits (default: about a second)
+    int withhold_next;          // self test of the bounded waits: applies to the next attention call only
     void* dev_blob;             // one allocation holding every device array
     hat::DevicePlan dev;
 };

@@ -256,3 +256,41 @@ def test_host_buffer_entry_point(cuda_device):
     assert_parity(lse.numpy(), want[0][1], "host entry lse")
     gk, gv = cache.pools_to_host()
     assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+
+
+def test_bounded_wait_gives_up_and_the_context_stays_usable(cuda_device):
+    """Failure detection without a fault: the tile kernel's producer withholds one transfer, the waiting
+    warps give up after the (shortened) bound, the status word reports it, and the next call is correct."""
+    from paper_2503_18989_b200 import binding as B, runner
+    sc = _manual("fp16", 2, 128, [300], [200], 21)
+    st = sc.steps[0]
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    assert ds.info["prefill_kernel"] == 1
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    B.hat_plan_set_wait_limit(ds.plan, 20_000_000, withhold_next_call=True)      # about 10 ms
+    ds.attend(fused_append=True)
+    assert B.hat_last_device_status(ds.plan) == B.HAT_ERR_DEVICE_TIMEOUT
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK                            # reading clears the word
+    B.hat_plan_set_wait_limit(ds.plan, 0)
+    ds.attend(fused_append=True)                                                    # the self test was one-shot
+    go, gl = ds.results()
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    kp, vp, want = oracle_replay(sc)
+    assert_parity(go, want[0][0], "out after a timed-out call")
+    assert_parity(gl, want[0][1], "lse after a timed-out call")
+
+
+def test_long_prefill_request_is_cut_into_at_most_32_key_ranges(cuda_device):
+    from paper_2503_18989_b200 import binding as B, runner
+    sc = _manual("fp16", 1, 128, [20000], [300], 22)
+    cache, got = _run(sc, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert 1 < ds.info["max_splits"] <= 32 and ds.info["num_merge_rows"] == 300
+    rng = np.random.default_rng(0)
+    samples = np.asarray([(0, int(i), 0) for i in [0, 127, 128, 255, 256, 299, *rng.integers(0, 300, 20)]], np.int64)
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(sc.cache, kp, vp, sc.steps[0])
+    wo, wl = O.attention_rows(sc.cache, kp, vp, sc.steps[0], samples)
+    assert_parity(got[0][0][samples[:, 1], 0], wo, "long prefill out")
+    assert_parity(got[0][1][samples[:, 1], 0], wl, "long prefill lse")
