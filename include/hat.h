@@ -121,6 +121,8 @@ typedef struct hat_plan_info {
     int64_t workspace_bytes;
     int64_t attn_flops;          /* 4*d*H*sum_r [C_r*P_r + C_r*(C_r+1)/2] */
     int64_t kv_read_bytes;       /* 2*sum_r (P_r+C_r)*H*d*elem: every visible K and V row read once per head */
+    int32_t stream_kernel;       /* 0 = cp.async streaming kernel, 1 = TMA streaming kernel */
+    int32_t reserved;
 } hat_plan_info;
 
 const char* hat_status_string(int status);

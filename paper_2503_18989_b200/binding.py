@@ -60,7 +60,8 @@ class hat_plan_info(C.Structure):
                 ("num_prefill_items", C.c_int32), ("num_merge_rows", C.c_int32), ("max_splits", C.c_int32),
                 ("verify_split_len", C.c_int32), ("prefill_split_len", C.c_int32),
                 ("prefill_tile_rows", C.c_int32), ("prefill_kernel", C.c_int32),
-                ("workspace_bytes", C.c_int64), ("attn_flops", C.c_int64), ("kv_read_bytes", C.c_int64)]
+                ("workspace_bytes", C.c_int64), ("attn_flops", C.c_int64), ("kv_read_bytes", C.c_int64),
+                ("stream_kernel", C.c_int32), ("reserved", C.c_int32)]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

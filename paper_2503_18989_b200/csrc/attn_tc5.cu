@@ -20,6 +20,7 @@
 #include <cuda_fp16.h>
 
 #include "hat_internal.h"
+#include "tma_desc.h"
 
 namespace hat {
 namespace {
@@ -473,37 +474,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-bool encode_pool_map(CUtensorMap* map, bool bf16, const void* pool, int num_pages, int H, int64_t stride_page,
-                     int64_t stride_token, int64_t stride_head) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)kPageSize, (cuuint64_t)H, (cuuint64_t)num_pages};
-    const cuuint64_t strides[3] = {(cuuint64_t)stride_token * 2, (cuuint64_t)stride_head * 2, (cuuint64_t)stride_page * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(pool),
-              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 bool encode_q_map(CUtensorMap* map, bool bf16, const void* q, int T, int H) {
-    EncodeTiledFn fn = encode_fn();
+    EncodeTiledFn fn = tma_encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)T};
     const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)H * kD * 2};
@@ -521,18 +493,18 @@ bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t
     if (head_dim != kD || num_pages <= 0) return false;
     CUtensorMap m;
     // the encoder checks alignment and ranges only; any 16-byte aligned address will do for the probe
-    return encode_pool_map(&m, dtype == HAT_DTYPE_BF16, reinterpret_cast<const void*>(uintptr_t(1) << 30), num_pages, H,
-                           stride_page, stride_token, stride_head);
+    return tma_encode_pool_map(&m, dtype == HAT_DTYPE_BF16, reinterpret_cast<const void*>(uintptr_t(1) << 30), kD, num_pages,
+                               H, stride_page, stride_token, stride_head);
 }
 
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     CUtensorMap mq, mk, mv;
     if (!encode_q_map(&mq, bf16, args.q, plan->total_rows, plan->num_heads) ||
-        !encode_pool_map(&mk, bf16, args.cache.k_pool, plan->num_pages, plan->num_heads, args.cache.stride_page,
-                         args.cache.stride_token, args.cache.stride_head) ||
-        !encode_pool_map(&mv, bf16, args.cache.v_pool, plan->num_pages, plan->num_heads, args.cache.stride_page,
-                         args.cache.stride_token, args.cache.stride_head))
+        !tma_encode_pool_map(&mk, bf16, args.cache.k_pool, kD, plan->num_pages, plan->num_heads, args.cache.stride_page,
+                             args.cache.stride_token, args.cache.stride_head) ||
+        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, kD, plan->num_pages, plan->num_heads, args.cache.stride_page,
+                             args.cache.stride_token, args.cache.stride_head))
         return cudaErrorInvalidValue;
     const dim3 grid(plan->num_heads, (unsigned)plan->prefill_items.size());
     cudaError_t e;

@@ -346,6 +346,14 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
                                        cache->stride_token, cache->stride_head);
     schedule(p, num_sms, use_tc5);
+    // the streaming kernel takes its pages by TMA when a descriptor can be built for the pool layout
+    bool stream_tma = true;
+    if (const char* k = std::getenv("HAT_STREAM_KERNEL"))
+        if (std::strcmp(k, "mma") == 0) stream_tma = false;
+    if (stream_tma && !p->host_only)
+        stream_tma = stream_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
+                                             cache->stride_token, cache->stride_head);
+    p->info.stream_kernel = stream_tma ? 1 : 0;
 
     if (!p->host_only) {
         st = upload(p);
@@ -452,7 +460,8 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
     }
     mark(2);
     if (!plan->verify_items.empty()) {
-        e = launch_attn_mma(plan, a, /*verify_class=*/true, s);
+        e = plan->info.stream_kernel == 1 ? launch_attn_stream(plan, a, s)
+                                          : launch_attn_mma(plan, a, /*verify_class=*/true, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ran(2);
     }

@@ -105,5 +105,9 @@ cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, cudaStream_
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                           int64_t stride_head);
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+// TMA-fed streaming kernel: whether a TMA descriptor can be built for this pool layout, and the launcher
+bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
+                             int64_t stride_head);
+cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
 void count_launch(int n = 1);
 }  // namespace hat
