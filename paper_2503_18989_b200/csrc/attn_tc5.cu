@@ -1,23 +1,29 @@
 // Prefill-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
 //
-// One CTA = up to 256 query rows (two 128-row query tiles) of one request x one head x one key range; both query
-// tiles use the same K/V tiles in shared memory, and while one tile's softmax runs the tensor pipe works for the
-// other.  Roles:
-//   warp 0      TMA producer: Q tile once, then K and V tiles of 128 keys (8 pages x 2 halves of 64 columns,
-//               128-byte swizzle) into a two-slot K ring and a three-slot V ring, completion on mbarriers
+// Persistent kernel, one CTA per SM.  A work unit = up to 256 query rows (two 128-row query tiles) of one request x
+// one head x one key range; CTAs draw units (longest first) from a global counter until none is left.  Both query
+// tiles of a unit use the same K/V tiles in shared memory, and while one tile's softmax runs the tensor pipe works
+// for the other.  Roles:
+//   warp 0      draws the next unit and publishes it to the other roles; TMA producer: the unit's Q tiles, then K
+//               and V tiles of 128 keys (8 pages x 2 halves of 64 columns, 128-byte swizzle) into a two-slot K ring
+//               and a three-slot V ring, completion on mbarriers.  It runs ahead across units: the next unit's Q and
+//               first K/V tiles are already landing while the current unit's last tiles and its output are processed
 //   warp 1      one thread issues tcgen05.mma: S_t = Q_t K^T for query tile t, then O_t += P_t V with P read
 //               from TMEM; tcgen05.commit signals the consumers and frees the ring slots.  Owns the TMEM allocation
-//   warps 2-5, 6-9   one warpgroup per query tile, thread = query row = TMEM lane: tcgen05.ld of S, scale/mask/online softmax in
-//               registers (running maximum only moved when it grows by more than 2^8, so O is rarely rescaled),
-//               P written back to TMEM as the 16-bit A operand, final O / l and log-sum-exp to global memory
+//   warps 2-5, 6-9   one warpgroup per query tile, thread = query row = TMEM lane: tcgen05.ld of S, scale/mask/online
+//               softmax in registers (reference maximum only moved when it grows by more than 2^8, so O is rarely
+//               rescaled), P written back to TMEM as the 16-bit A operand; at the end of a unit O is pulled into
+//               registers (which frees the accumulator for the next unit), divided by l and stored with the lse
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512).  P_t(j) overwrites S_t(j) in place (16-bit pairs in
 // columns [0,64), the bf16 rounding remainder in [64,128)); S_t(j+1) is issued after P_t V(j) by the same thread, and
 // tcgen05 executes one thread's MMAs in issue order, so no extra barrier guards the reuse.
-// Every wait is bounded (about a second by default); a wait that gives up sets the plan's status word, raises a CTA-wide abort
-// flag that all other waits observe, and the CTA still frees its TMEM and exits normally.
+// Every wait is bounded (about a second by default); a wait that gives up sets the plan's status word, raises a
+// CTA-wide abort flag that all other waits observe, and the CTA still frees its TMEM and exits normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+
+#include <algorithm>
 
 #include "hat_internal.h"
 #include "tma_desc.h"
@@ -36,14 +42,16 @@ constexpr uint32_t kPageBoxBytes = 16 * 64 * 2;          // 2 KiB: one TMA box (
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
 
 struct __align__(8) Barriers {
-    uint64_t q_full;
+    uint64_t q_full, q_empty;
     uint64_t k_full[kStagesK], k_empty[kStagesK];
     uint64_t v_full[kStagesV], v_empty[kStagesV];
-    uint64_t s_full[2], p_ready[2], o_done[2];   // per query tile
+    uint64_t s_full[2], p_ready[2], o_done[2], o_free[2];   // per query tile
+    uint64_t unit_full[2], unit_empty[2];                   // two-slot queue of work units, producer -> other roles
     uint64_t drain;
-    long long wait_cycles;                       // bound of every wait below
+    long long wait_cycles;                                  // bound of every wait below
     uint32_t tmem_base;
     volatile int abort_flag;
+    volatile int unit_slot[2];                              // unit index, or -1 when the work has run out
 };
 constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + kStagesK + kStagesV) + 256;
 constexpr int kThreads = 320;   // producer warp, MMA warp, two softmax warpgroups
@@ -167,10 +175,35 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     }
 }
 
+// What every role needs to know about a unit; all of them decode it the same way.
+struct Unit {
+    int h, r, P, C, row_base, row0, kv_begin, kv_end, part;
+    int nq;       // query tiles in use (1 or 2)
+    int n_all;    // key tiles of the range
+    int n_q0;     // key tiles query tile 0 can see (tile 0 does not see the keys past its own last row)
+};
+__device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* __restrict__ items, int unit) {
+    const int H = a.plan.num_heads;
+    const WorkItem it = items[unit / H];
+    Unit u;
+    u.h = unit % H;
+    u.r = it.req;
+    u.P = a.plan.prefix_len[u.r];
+    u.C = a.plan.chunk_len[u.r];
+    u.row_base = a.plan.cu_chunk[u.r];
+    u.row0 = it.row0; u.kv_begin = it.kv_begin; u.kv_end = it.kv_end; u.part = it.part;
+    u.nq = (u.C - u.row0 > kRows) ? 2 : 1;
+    u.n_all = (u.kv_end - u.kv_begin + kKeys - 1) / kKeys;
+    const int end0 = min(u.kv_end, u.P + u.row0 + kRows);
+    u.n_q0 = u.nq == 1 ? u.n_all : max(0, (end0 - u.kv_begin + kKeys - 1) / kKeys);
+    return u;
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_constant__ CUtensorMap map_q,
-                const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units, int32_t* work_counter,
+                const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle pattern and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -179,29 +212,21 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
     unsigned char* v_ring = k_ring + kStagesK * kTileBytes;
     Barriers* bars = reinterpret_cast<Barriers*>(v_ring + kStagesV * kTileBytes);
 
-    const WorkItem item = items[blockIdx.y];
-    const int h = blockIdx.x;
     const int H = a.plan.num_heads;
-    const int r = item.req;
-    const int P = a.plan.prefix_len[r];
-    const int C = a.plan.chunk_len[r];
-    const int row_base = a.plan.cu_chunk[r];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // the item's rows form up to two 128-row query tiles; tile 0 does not see the keys past its own last row
-    const int nq = (C - item.row0 > kRows) ? 2 : 1;
-    const int n_all = (item.kv_end - item.kv_begin + kKeys - 1) / kKeys;
-    const int end0 = min(item.kv_end, P + item.row0 + kRows);
-    const int n_q0 = nq == 1 ? n_all : max(0, (end0 - item.kv_begin + kKeys - 1) / kKeys);
     int32_t* status = a.plan.status;
 
     if (threadIdx.x == 0) {
-        mbar_init(&bars->q_full, 1);
+        mbar_init(&bars->q_full, 1); mbar_init(&bars->q_empty, 1);
         for (int s = 0; s < kStagesK; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
         for (int s = 0; s < kStagesV; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars->s_full[s], 1);
             mbar_init(&bars->p_ready[s], 128);
             mbar_init(&bars->o_done[s], 1);
+            mbar_init(&bars->o_free[s], 128);
+            mbar_init(&bars->unit_full[s], 1);
+            mbar_init(&bars->unit_empty[s], 1 + 256);            // the MMA thread and every softmax thread
         }
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
@@ -219,39 +244,62 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
     const uint32_t tmem = bars->tmem_base;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        const int32_t* __restrict__ table = a.plan.block_table + (int64_t)r * a.plan.max_pages;
-        if (lane == 0) mbar_expect_tx(&bars->q_full, nq * kTileBytes);
-        __syncwarp();
-        if (lane < 2 * nq)      // lane = 2 * (query tile) + (column half)
-            tma_load_3d(smem_u32(q_tiles) + (lane >> 1) * kTileBytes + (lane & 1) * kSlabBytes, &map_q, (lane & 1) * 64, h,
-                        row_base + item.row0 + (lane >> 1) * kRows, &bars->q_full);
+        // ------------------------------------------------------------------ unit fetch + TMA producer
         // lane l < 16 moves box (page l/2 of the tile, column half l%2)
         const int pg = lane >> 1, half = lane & 1;
+        int kt = 0;                                              // K/V tiles issued so far, over all units
         bool ok = true;
-        for (int j = 0; j < n_all; ++j) {
-            const int sk = j % kStagesK, sv = j % kStagesV;
-            const int kb = item.kv_begin + j * kKeys;
-            const int npages = (min(item.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
-            int page = 0;
-            if (lane < 16 && pg < npages) page = __ldg(table + kb / kPageSize + pg);
-            if (j >= kStagesK) ok = mbar_wait(&bars->k_empty[sk], ((j / kStagesK) & 1) ^ 1, bars, status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (lane == 0) mbar_expect_tx(&bars->k_full[sk], npages * 2 * kPageBoxBytes);
+        for (int un = 0; ok; ++un) {
+            const int slot = un & 1;
+            if (un >= 2) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->unit_empty[slot], ((un >> 1) - 1) & 1, bars, status));
+                if (!ok) break;
+            }
+            int unit = 0;
+            if (lane == 0) {
+                unit = atomicAdd(work_counter, 1);
+                if (unit >= total_units) unit = -1;
+                bars->unit_slot[slot] = unit;
+                mbar_arrive(&bars->unit_full[slot]);             // release: the slot is written before the arrival
+            }
+            unit = __shfl_sync(0xffffffffu, unit, 0);
+            if (unit < 0) break;
+            const Unit u = decode_unit(a, items, unit);
+            const int32_t* __restrict__ table = a.plan.block_table + (int64_t)u.r * a.plan.max_pages;
+            // Q tiles: the previous unit's last S must have read the old ones
+            if (un > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->q_empty, (un - 1) & 1, bars, status));
+                if (!ok) break;
+            }
+            if (lane == 0) mbar_expect_tx(&bars->q_full, u.nq * kTileBytes);
             __syncwarp();
-            if (lane < 16 && pg < npages)
-                tma_load_4d(smem_u32(k_ring) + sk * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0, h,
-                            page, &bars->k_full[sk]);
-            if (j >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((j / kStagesV) & 1) ^ 1, bars, status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (a.withhold && j == 0) continue;          // self test: this V tile never arrives, its consumers give up
-            if (lane == 0) mbar_expect_tx(&bars->v_full[sv], npages * 2 * kPageBoxBytes);
-            __syncwarp();
-            if (lane < 16 && pg < npages)
-                tma_load_4d(smem_u32(v_ring) + sv * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0, h,
-                            page, &bars->v_full[sv]);
+            if (lane < 2 * u.nq)      // lane = 2 * (query tile) + (column half)
+                tma_load_3d(smem_u32(q_tiles) + (lane >> 1) * kTileBytes + (lane & 1) * kSlabBytes, &map_q, (lane & 1) * 64, u.h,
+                            u.row_base + u.row0 + (lane >> 1) * kRows, &bars->q_full);
+            for (int j = 0; j < u.n_all; ++j, ++kt) {
+                const int sk = kt % kStagesK, sv = kt % kStagesV;
+                const int kb = u.kv_begin + j * kKeys;
+                const int npages = (min(u.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
+                int page = 0;
+                if (lane < 16 && pg < npages) page = __ldg(table + kb / kPageSize + pg);
+                if (kt >= kStagesK) ok = mbar_wait(&bars->k_empty[sk], ((kt / kStagesK) & 1) ^ 1, bars, status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(&bars->k_full[sk], npages * 2 * kPageBoxBytes);
+                __syncwarp();
+                if (lane < 16 && pg < npages)
+                    tma_load_4d(smem_u32(k_ring) + sk * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0,
+                                u.h, page, &bars->k_full[sk]);
+                if (kt >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((kt / kStagesV) & 1) ^ 1, bars, status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (a.withhold && kt == 0) continue;         // self test: this V tile never arrives, its consumers give up
+                if (lane == 0) mbar_expect_tx(&bars->v_full[sv], npages * 2 * kPageBoxBytes);
+                __syncwarp();
+                if (lane < 16 && pg < npages)
+                    tma_load_4d(smem_u32(v_ring) + sv * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0,
+                                u.h, page, &bars->v_full[sv]);
+            }
         }
         if (!ok) {
             // give copies already in flight a bounded chance to land before the CTA's shared memory is released
@@ -264,62 +312,90 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
             constexpr uint32_t fmt = BF16 ? 1u : 0u;
             constexpr uint32_t idesc_s = make_idesc(fmt, 0, kRows, kKeys);   // Q (K-major) x K (K-major)
             constexpr uint32_t idesc_o = make_idesc(fmt, 1, kRows, kD);      // P (TMEM)    x V (MN-major)
-            bool ok = mbar_wait(&bars->q_full, 0, bars, status);
-            int k_ready = -1, v_ready = -1;                                  // last K / V tile known to have landed
-            // S_qt(j) = Q_qt K(j)^T into TMEM columns [128 qt, 128 qt + 128)
-            auto issue_s = [&](int qt, int j) {
-                const int st = j % kStagesK;
-                if (k_ready < j) {
-                    ok = mbar_wait(&bars->k_full[st], (j / kStagesK) & 1, bars, status);
-                    k_ready = j;
-                    if (!ok) return;
-                }
-                const uint32_t q_addr = smem_u32(q_tiles) + qt * kTileBytes;
-                const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
-                tc_fence_after();
+            bool ok = true;
+            int kt_base = 0;                          // K/V tiles of the units before this one
+            int p_cnt[2] = {0, 0};                    // completions of p_ready[t] consumed so far
+            int f_cnt[2] = {0, 0};                    // completions of o_free[t] consumed so far
+            bool o_busy[2] = {false, false};          // O_t holds a finished unit that its warpgroup may still be reading
+            for (int un = 0; ok; ++un) {
+                const int slot = un & 1;
+                ok = mbar_wait(&bars->unit_full[slot], (un >> 1) & 1, bars, status);
+                if (!ok) break;
+                const int unit = bars->unit_slot[slot];
+                mbar_arrive(&bars->unit_empty[slot]);
+                if (unit < 0) break;
+                const Unit u = decode_unit(a, items, unit);
+                ok = mbar_wait(&bars->q_full, un & 1, bars, status);
+                if (!ok) break;
+                int k_ready = -1, v_ready = -1;       // last K / V tile of this unit known to have landed
+                // S_t(j) = Q_t K(j)^T into TMEM columns [128 t, 128 t + 128)
+                auto issue_s = [&](int qt, int j) {
+                    const int kt = kt_base + j, st = kt % kStagesK;
+                    if (k_ready < j) {
+                        ok = mbar_wait(&bars->k_full[st], (kt / kStagesK) & 1, bars, status);
+                        k_ready = j;
+                        if (!ok) return;
+                    }
+                    const uint32_t q_addr = smem_u32(q_tiles) + qt * kTileBytes;
+                    const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < kD / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
-                    mma_ss(tmem + qt * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
-                }
-                tc_commit(&bars->s_full[qt]);
-                if (qt == nq - 1) tc_commit(&bars->k_empty[st]);             // the last reader of this K tile
-            };
-            // O_qt (+)= P_qt(j) V(j); P sits in the columns S_qt(j) was computed in
-            auto issue_pv = [&](int qt, int j) {
-                const int st = j % kStagesV;
-                if (v_ready < j) {
-                    ok = mbar_wait(&bars->v_full[st], (j / kStagesV) & 1, bars, status);
-                    v_ready = j;
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
+                        mma_ss(tmem + qt * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                    }
+                    tc_commit(&bars->s_full[qt]);
+                    if (qt == u.nq - 1) {
+                        tc_commit(&bars->k_empty[st]);                       // the last reader of this K tile
+                        if (j == u.n_all - 1) tc_commit(&bars->q_empty);     // and the unit's last read of the Q tiles
+                    }
+                };
+                // O_t (+)= P_t(j) V(j); P sits in the columns S_t(j) was computed in
+                auto issue_pv = [&](int qt, int j) {
+                    const int kt = kt_base + j, st = kt % kStagesV;
+                    if (v_ready < j) {
+                        ok = mbar_wait(&bars->v_full[st], (kt / kStagesV) & 1, bars, status);
+                        v_ready = j;
+                        if (!ok) return;
+                    }
+                    if (j == 0 && o_busy[qt]) {
+                        // the accumulator still holds the previous unit: wait until its rows are in registers
+                        ok = mbar_wait(&bars->o_free[qt], f_cnt[qt] & 1, bars, status);
+                        ++f_cnt[qt];
+                        if (!ok) return;
+                    }
+                    ok = mbar_wait(&bars->p_ready[qt], p_cnt[qt] & 1, bars, status);
+                    ++p_cnt[qt];
                     if (!ok) return;
-                }
-                ok = mbar_wait(&bars->p_ready[qt], j & 1, bars, status);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
-                const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
+                    tc_fence_after();
+                    const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
+                    const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
 #pragma unroll
-                for (int ks = 0; ks < kKeys / 16; ++ks) {
-                    // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
-                    const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
-                    mma_ts(to, tp + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));
-                    if constexpr (BF16) mma_ts(to, tp + 64 + ks * 8, vdesc, idesc_o, true);
+                    for (int ks = 0; ks < kKeys / 16; ++ks) {
+                        // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
+                        const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
+                        mma_ts(to, tp + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));
+                        if constexpr (BF16) mma_ts(to, tp + 64 + ks * 8, vdesc, idesc_o, true);
+                    }
+                    tc_commit(&bars->o_done[qt]);
+                    if (qt == u.nq - 1) tc_commit(&bars->v_empty[st]);
+                };
+                if (u.n_q0 > 0) issue_s(0, 0);
+                if (ok && u.nq == 2) issue_s(1, 0);
+                for (int j = 0; j < u.n_all && ok; ++j) {
+                    // tile 0's P V(j), then at once its next S: the tensor pipe works on them while tile 1's softmax runs
+                    if (j < u.n_q0) {
+                        issue_pv(0, j);
+                        if (ok && j + 1 < u.n_q0) issue_s(0, j + 1);
+                    }
+                    if (ok && u.nq == 2) {
+                        issue_pv(1, j);
+                        if (ok && j + 1 < u.n_all) issue_s(1, j + 1);
+                    }
                 }
-                tc_commit(&bars->o_done[qt]);
-                if (qt == nq - 1) tc_commit(&bars->v_empty[st]);
-            };
-            if (ok && n_q0 > 0) issue_s(0, 0);
-            if (ok && nq == 2) issue_s(1, 0);
-            for (int j = 0; j < n_all && ok; ++j) {
-                // tile 0's P V(j), then at once its next S: the tensor pipe works on them while tile 1's softmax runs
-                if (j < n_q0) {
-                    issue_pv(0, j);
-                    if (ok && j + 1 < n_q0) issue_s(0, j + 1);
-                }
-                if (ok && nq == 2) {
-                    issue_pv(1, j);
-                    if (ok && j + 1 < n_all) issue_s(1, j + 1);
-                }
+                o_busy[0] = u.n_q0 > 0;
+                if (u.nq == 2) o_busy[1] = true;
+                kt_base += u.n_all;
             }
             if (!ok) {
                 // gave up: let the MMAs already issued finish (bounded) before TMEM is released
@@ -330,138 +406,152 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_con
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ softmax / correction / epilogue
+        // ------------------------------------------------------------------ softmax / correction / output
         const int qt = (warp - 2) >> 2;                     // query tile of this warpgroup
         const int quarter = warp & 3;                       // TMEM lanes this warp may touch
         const int t = quarter * 32 + lane;                  // query row inside the tile = TMEM lane
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
         const uint32_t tm_s = tmem + qt * 128 + lane_sel, tm_o = tmem + 256 + qt * 128 + lane_sel;
-        const int n_mine = (qt == 0) ? n_q0 : n_all;
-        const int i_row = item.row0 + qt * kRows + t;       // row inside the chunk
-        const int last_key = min(P + i_row, item.kv_end - 1);
         const int wg_tid = (int)threadIdx.x - 64 - qt * 128;
-        float m_used = -INFINITY, l = 0.f;                  // in units of scale_log2
         const float sc = a.scale_log2;
+        int kt_base = 0;                                    // K/V tiles of the units before this one
+        int s_cnt = 0, o_cnt = 0;                           // completions of s_full[qt] / o_done[qt] consumed so far
         bool ok = true;
-        if (qt < nq) {
-            for (int j = 0; j < n_mine; ++j) {
-                const int kb = item.kv_begin + j * kKeys;
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[qt], j & 1, bars, status));
-                if (!ok) break;
-                tc_fence_after();
-                float s[kKeys];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
-                tmem_ld_wait();
-
-                // raw maximum (the scale is positive, so it commutes with max); four independent chains
-                const int lim = last_key - kb;              // keys 0..lim of this tile are visible to this row
-                if (lim < kKeys - 1) {
-#pragma unroll
-                    for (int k = 0; k < kKeys; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
-                }
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                for (int k = 0; k < kKeys; k += 8) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], fmaxf(s[k + 2 * u], s[k + 2 * u + 1]));
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
-                // move the reference maximum only when it grew by more than the threshold
-                float alpha = 1.f;
-                bool rescale = false;
-                if (mx > m_used + kRescaleThreshold) {
-                    alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
-                    rescale = (m_used != -INFINITY);
-                    m_used = mx;
-                }
-                const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
-                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t p[16];
-                    uint32_t pl[16];
-#pragma unroll
-                    for (int k = 0; k < 32; k += 2) {
-                        const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
-                        const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
-                        sum4[(k >> 1) & 3] += e0 + e1;
-                        p[k / 2] = pack2<BF16>(e0, e1);
-                        if constexpr (BF16) {
-                            const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
-                            const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
-                            pl[k / 2] = pack2<BF16>(r0, r1);
-                        }
-                    }
-                    tmem_st16(tm_s + c * 16, p);
-                    if constexpr (BF16) tmem_st16(tm_s + 64 + c * 16, pl);
-                }
-                l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-
-                // O may only be rescaled once the previous P V product has finished; waiting here every tile (it
-                // has long completed by now) also keeps this thread's view of the barrier phase in step
-                if (j > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], (j - 1) & 1, bars, status));
+        for (int un = 0; ok; ++un) {
+            const int slot = un & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars->unit_full[slot], (un >> 1) & 1, bars, status));
+            if (!ok) break;
+            const int unit = bars->unit_slot[slot];
+            mbar_arrive(&bars->unit_empty[slot]);
+            if (unit < 0) break;
+            const Unit u = decode_unit(a, items, unit);
+            if (qt < u.nq) {
+                const int n_mine = (qt == 0) ? u.n_q0 : u.n_all;
+                const int i_row = u.row0 + qt * kRows + t;   // row inside the chunk
+                const int last_key = min(u.P + i_row, u.kv_end - 1);
+                float m_used = -INFINITY, l = 0.f;           // in units of scale_log2
+                for (int j = 0; j < n_mine; ++j) {
+                    const int kb = u.kv_begin + j * kKeys;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[qt], s_cnt & 1, bars, status));
+                    ++s_cnt;
                     if (!ok) break;
                     tc_fence_after();
-                }
-                if (__any_sync(0xffffffffu, rescale)) {
+                    float s[kKeys];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
+                    tmem_ld_wait();
+
+                    // raw maximum (the scale is positive, so it commutes with max); four independent chains
+                    const int lim = last_key - kb;          // keys 0..lim of this tile are visible to this row
+                    if (lim < kKeys - 1) {
+#pragma unroll
+                        for (int k = 0; k < kKeys; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
+                    }
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int k = 0; k < kKeys; k += 8) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], fmaxf(s[k + 2 * v], s[k + 2 * v + 1]));
+                    }
+                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
+                    // move the reference maximum only when it grew by more than the threshold
+                    float alpha = 1.f;
+                    bool rescale = false;
+                    if (mx > m_used + kRescaleThreshold) {
+                        alpha = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - mx);
+                        rescale = (m_used != -INFINITY);
+                        m_used = mx;
+                    }
+                    const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
+                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tm_o + c * 32, o);
-                        tmem_ld_wait();
+                        uint32_t p[16];
+                        uint32_t pl[16];
 #pragma unroll
-                        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                        tmem_st32(tm_o + c * 32, o);
+                        for (int k = 0; k < 32; k += 2) {
+                            const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
+                            const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
+                            sum4[(k >> 1) & 3] += e0 + e1;
+                            p[k / 2] = pack2<BF16>(e0, e1);
+                            if constexpr (BF16) {
+                                const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
+                                const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
+                                pl[k / 2] = pack2<BF16>(r0, r1);
+                            }
+                        }
+                        tmem_st16(tm_s + c * 16, p);
+                        if constexpr (BF16) tmem_st16(tm_s + 64 + c * 16, pl);
                     }
+                    l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+
+                    // O may only be rescaled once the previous P V product has finished; waiting here every tile (it
+                    // has long completed by now) also keeps this thread's count of the barrier's phases exact
+                    if (j > 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], o_cnt & 1, bars, status));
+                        ++o_cnt;
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
+                    if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tm_o + c * 32, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                            tmem_st32(tm_o + c * 32, o);
+                        }
+                    }
+                    tmem_st_wait();
+                    // a range that ends inside this tile: V rows past the range were not loaded (or hold stale
+                    // slots); zero them so that 0 * garbage cannot produce NaN (both warpgroups may do it: same zeros)
+                    if (kb + kKeys > u.kv_end) {
+                        const int kt = kt_base + j;
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[kt % kStagesV], (kt / kStagesV) & 1, bars, status));
+                        if (!ok) break;
+                        unsigned char* vt = v_ring + (kt % kStagesV) * kTileBytes;
+                        const int first = u.kv_end - kb;
+                        for (int idx = wg_tid; idx < (kKeys - first) * 16; idx += 128) {
+                            const int row = first + idx / 16, part = idx % 16;     // 16 vectors of 16 bytes per 256-byte row
+                            *reinterpret_cast<uint4*>(vt + (part >> 3) * kSlabBytes + row * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    }
+                    tc_fence_before();
+                    mbar_arrive(&bars->p_ready[qt]);
                 }
-                tmem_st_wait();
-                // a range that ends inside this tile: V rows past the range were not loaded (or hold stale
-                // slots); zero them so that 0 * garbage cannot produce NaN (both warpgroups may do it: same zeros)
-                if (kb + kKeys > item.kv_end) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[j % kStagesV], (j / kStagesV) & 1, bars, status));
+                if (!ok) break;
+                // ---- output of the unit: pull O into registers, hand the accumulator back, then store
+                float o[kD];
+                if (n_mine > 0) {                            // uniform over the warpgroup
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], o_cnt & 1, bars, status));
+                    ++o_cnt;
                     if (!ok) break;
-                    unsigned char* vt = v_ring + (j % kStagesV) * kTileBytes;
-                    const int first = item.kv_end - kb;
-                    for (int idx = wg_tid; idx < (kKeys - first) * 16; idx += 128) {
-                        const int row = first + idx / 16, part = idx % 16;     // 16 vectors of 16 bytes per 256-byte row
-                        *reinterpret_cast<uint4*>(vt + (part >> 3) * kSlabBytes + row * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(tm_o + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    mbar_arrive(&bars->o_free[qt]);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < kD; ++k) o[k] = 0.f;
                 }
-                tc_fence_before();
-                mbar_arrive(&bars->p_ready[qt]);
-            }
-            if (ok && n_mine > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], (n_mine - 1) & 1, bars, status));
-            if (ok) {
-                tc_fence_after();
-                const float inv = l > 0.f ? 1.f / l : 0.f;
-                const bool valid = i_row < C;
-                float* obase; float* lbase; int64_t orow;
-                if (item.part < 0) { obase = a.out; lbase = a.lse; orow = row_base + i_row; }
-                else { obase = a.part_out; lbase = a.part_lse; orow = item.part + qt * kRows + t; }
-                float* dst = obase + (orow * H + h) * kD;
+                if (i_row < u.C) {
+                    const float inv = l > 0.f ? 1.f / l : 0.f;
+                    float* obase; float* lbase; int64_t orow;
+                    if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
+                    else { obase = a.part_out; lbase = a.part_lse; orow = u.part + qt * kRows + t; }
+                    float* dst = obase + (orow * H + u.h) * kD;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    if (n_mine > 0) {                       // uniform over the warpgroup
-                        tmem_ld32(tm_o + c * 32, o);
-                        tmem_ld_wait();
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) o[k] = 0u;
-                    }
-                    if (valid) {
-#pragma unroll
-                        for (int k = 0; k < 32; k += 4)
-                            *reinterpret_cast<float4*>(dst + c * 32 + k) =
-                                make_float4(__uint_as_float(o[k]) * inv, __uint_as_float(o[k + 1]) * inv,
-                                            __uint_as_float(o[k + 2]) * inv, __uint_as_float(o[k + 3]) * inv);
-                    }
+                    for (int k = 0; k < kD; k += 4)
+                        *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
+                    lbase[orow * H + u.h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
                 }
-                if (valid) lbase[orow * H + h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
             }
+            kt_base += u.n_all;
         }
     }
 
@@ -506,16 +596,20 @@ cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStre
         !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, kD, plan->num_pages, plan->num_heads, args.cache.stride_page,
                              args.cache.stride_token, args.cache.stride_head))
         return cudaErrorInvalidValue;
-    const dim3 grid(plan->num_heads, (unsigned)plan->prefill_items.size());
-    cudaError_t e;
+    // one CTA per SM draws (item, head) units from a counter that is cleared on the stream first
+    const int total_units = (int)plan->prefill_items.size() * plan->num_heads;
+    int32_t* counter = plan->dev.status + 1;
+    cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(int32_t), stream);
+    if (e != cudaSuccess) return e;
+    const dim3 grid((unsigned)std::min(total_units, plan->num_sms));
     if (bf16) {
         e = cudaFuncSetAttribute(attn_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_tc5_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
+        attn_tc5_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, mq, mk, mv);
     } else {
         e = cudaFuncSetAttribute(attn_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_tc5_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, mq, mk, mv);
+        attn_tc5_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, mq, mk, mv);
     }
     count_launch();
     return cudaGetLastError();

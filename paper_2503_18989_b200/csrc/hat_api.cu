@@ -345,6 +345,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     if (use_tc5 && !p->host_only)
         use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
                                        cache->stride_token, cache->stride_head);
+    p->num_sms = num_sms;
     schedule(p, num_sms, use_tc5);
     // the streaming kernel takes its pages by TMA when a descriptor can be built for the pool layout
     bool stream_tma = true;

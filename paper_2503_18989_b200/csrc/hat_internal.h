@@ -83,6 +83,7 @@ struct hat_plan {
     int32_t dtype, num_pages, num_heads, head_dim, max_pages, num_requests, total_rows;
     bool host_only;
     int device;
+    int num_sms;
     std::vector<int32_t> cu_chunk, prefix_len, chunk_len, block_table, row_req;
     std::vector<hat::WorkItem> verify_items, prefill_items;
     std::vector<hat::MergeRow> merge_rows;
