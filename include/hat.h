@@ -143,7 +143,8 @@ int64_t     hat_launch_count(void);
  * Unless HAT_PLAN_HOST_ONLY is set the schedule is uploaded to the current
  * device (one cudaMalloc + one synchronous copy).  A plan can be reused for
  * every layer of the step and must be destroyed with hat_plan_destroy.
- * Errors: INVALID_ARG, UNSUPPORTED, OUT_OF_RANGE, CUDA.  *out is NULL on error.
+ * Errors: INVALID_ARG, UNSUPPORTED, OUT_OF_RANGE, CUDA, TOO_LARGE (more than 65535 work items of one class,
+ * i.e. key ranges or 256-row tiles, in one batch).  *out is NULL on error.
  */
 int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, hat_plan** out);
 int hat_plan_get_info(const hat_plan* plan, hat_plan_info* out);

@@ -355,6 +355,12 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         stream_tma = stream_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
                                              cache->stride_token, cache->stride_head);
     p->info.stream_kernel = stream_tma ? 1 : 0;
+    // launch-geometry limits: work items index gridDim.y (65535), partial rows and units are 32-bit
+    if (p->verify_items.size() > 65535 || p->prefill_items.size() > 65535 || p->num_heads > 65535 ||
+        p->part_rows > INT32_MAX / 2 || (int64_t)p->prefill_items.size() * p->num_heads > INT32_MAX / 2) {
+        delete p;
+        return HAT_ERR_TOO_LARGE;
+    }
 
     if (!p->host_only) {
         st = upload(p);

@@ -162,3 +162,12 @@ def test_long_request_never_exceeds_32_key_ranges(hat_lib):
     p = _plan(c, [n], [4], table)
     info = B.hat_plan_get_info(p).as_dict()
     assert info["max_splits"] <= 32 and info["num_verify_items"] == info["max_splits"]
+
+
+def test_batches_beyond_the_launch_limits_are_rejected(hat_lib):
+    # 70000 one-token requests = 70000 streaming work items: more than one grid dimension can index
+    n = 70000
+    c = _cache(num_pages=n, H=1, d=64)
+    table = np.arange(n, dtype=np.int32)[:, None]
+    assert _status(_plan, c, np.zeros(n, np.int32), np.ones(n, np.int32), table, H=1) == B.HAT_ERR_TOO_LARGE
+    assert _status(_plan, c, np.zeros(60000, np.int32), np.ones(60000, np.int32), table[:60000], H=1) == B.HAT_OK
