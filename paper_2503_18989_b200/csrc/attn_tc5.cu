@@ -222,11 +222,11 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
         for (int s = 0; s < kStagesV; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars->s_full[s], 1);
-            mbar_init(&bars->p_ready[s], 128);
+            mbar_init(&bars->p_ready[s], 4);                     // one arrival per softmax warp
             mbar_init(&bars->o_done[s], 1);
-            mbar_init(&bars->o_free[s], 128);
+            mbar_init(&bars->o_free[s], 4);
             mbar_init(&bars->unit_full[s], 1);
-            mbar_init(&bars->unit_empty[s], 1 + 256);            // the MMA thread and every softmax thread
+            mbar_init(&bars->unit_empty[s], 1 + 8);              // the MMA thread and every softmax warp
         }
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
@@ -422,7 +422,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
             ok = __all_sync(0xffffffffu, mbar_wait(&bars->unit_full[slot], (un >> 1) & 1, bars, status));
             if (!ok) break;
             const int unit = bars->unit_slot[slot];
-            mbar_arrive(&bars->unit_empty[slot]);
+            __syncwarp();                                    // every lane has read the slot
+            if (lane == 0) mbar_arrive(&bars->unit_empty[slot]);
             if (unit < 0) break;
             const Unit u = decode_unit(a, items, unit);
             if (qt < u.nq) {
@@ -519,8 +520,10 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         }
                         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                     }
+                    // one arrival per warp: every lane's P is in TMEM (wait::st) and fenced before the warp meets
                     tc_fence_before();
-                    mbar_arrive(&bars->p_ready[qt]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->p_ready[qt]);
                 }
                 if (!ok) break;
                 // ---- output of the unit: pull O into registers, hand the accumulator back, then store
@@ -534,7 +537,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                     for (int c = 0; c < 4; ++c) tmem_ld32(tm_o + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
                     tmem_ld_wait();
                     tc_fence_before();
-                    mbar_arrive(&bars->o_free[qt]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->o_free[qt]);
                 } else {
 #pragma unroll
                     for (int k = 0; k < kD; ++k) o[k] = 0.f;
