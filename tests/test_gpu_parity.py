@@ -294,3 +294,24 @@ def test_long_prefill_request_is_cut_into_at_most_32_key_ranges(cuda_device):
     wo, wl = O.attention_rows(sc.cache, kp, vp, sc.steps[0], samples)
     assert_parity(got[0][0][samples[:, 1], 0], wo, "long prefill out")
     assert_parity(got[0][1][samples[:, 1], 0], wl, "long prefill lse")
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_small_batches(cuda_device, seed):
+    """Seeded random batches that mix every chunk class, odd prefixes, both types, both head sizes and both
+    layouts, with few heads so that the persistent tile kernel strings several units through one CTA and
+    key ranges get cut (few CTAs)."""
+    rng = np.random.Generator(np.random.PCG64(1000 + seed))
+    dtype = ["fp16", "bf16"][seed % 2]
+    d = [128, 128, 64][seed % 3]
+    H = int(rng.integers(1, 4))
+    R = int(rng.integers(1, 9))
+    kinds = rng.integers(0, 5, size=R)
+    chunk = np.where(kinds == 0, rng.integers(0, 3, size=R),                 # empty / one or two rows
+            np.where(kinds == 1, rng.integers(1, 17, size=R),                # streaming class
+            np.where(kinds == 2, rng.integers(17, 130, size=R),              # one query tile
+            np.where(kinds == 3, rng.integers(130, 300, size=R),             # two query tiles, ragged
+                     rng.integers(300, 700, size=R)))))                      # several 256-row items
+    prefix = np.where(rng.random(R) < 0.3, 0, rng.integers(0, 1500, size=R))
+    sc = _manual(dtype, H, d, prefix, chunk, 2000 + seed, layout=["paged", "contiguous"][(seed // 2) % 2])
+    _check_full(sc, cuda_device, fused_append=bool(seed % 2))
