@@ -427,6 +427,22 @@ def main():
             "kv_gbs": world * total["kv_bytes"] / (ms_per_step * 1e-3) / 1e9,
             "plan": steps[-1].info,
         }
+        # Close the paper's control loop on the measured delay (Sec. 3.2-3.3, 3.5): one observation of (batched token
+        # size, delay of this attention step), then the chunk size and parallel-drafting steps the controller would
+        # hand to a device with the paper's WiFi rates (7.5 MB/s up, 12.5 MB/s down, 20 ms per drafting step).
+        try:
+            ctrl = B.Ctrl(0.8, 64.0, 256, 1)
+            B.hat_ctrl_observe(ctrl, float(total["rows"]), ms_per_step * 1e-3)
+            B.hat_ctrl_device_observe(ctrl, 0, 0.020, 7.5e6, 12.5e6)
+            a_bytes = float(sc.cache.num_heads * sc.cache.head_dim * 2)
+            line["controller"] = {
+                "mu_tokens": B.hat_ctrl_mu(ctrl), "g_seconds": B.hat_ctrl_predict(ctrl, B.hat_ctrl_mu(ctrl)),
+                "chunk_size_eq3": B.hat_ctrl_chunk_size(ctrl, 0, a_bytes, 1, 16, 2048),
+                "parallel_draft_steps_eq6": B.hat_ctrl_parallel_draft_steps(ctrl, 0, 4, a_bytes),
+                "note": "g holds one observation of this attention step alone, not of a whole middle-submodel step"}
+            ctrl.close()
+        except Exception as exc:                     # the controller is a report item, never a reason to lose the line
+            line["controller"] = {"error": str(exc)}
         if not args.no_cpu_baseline and world == 1:
             rate, cores, sample, _, _ = time_oracle(sc, args.cpu_budget)
             line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",

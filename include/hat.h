@@ -242,6 +242,41 @@ int hat_last_device_status(const hat_plan* plan, void* stream, int* out);
 int hat_plan_set_wait_limit(hat_plan* plan, long long cycles, int withhold_next_call);
 
 /*
+ * Cloud-side control plane (host only; no CUDA call).  It closes the loop the
+ * paper describes around the attention step: per round the cloud records the
+ * batched token size and the in-cloud computation delay, keeps moving
+ * averages of them (Sec. 3.2, Eq. 1-2, alpha = 0.8 in the paper's
+ * experiments), and from the predicted delay g(.) derives each device's
+ * prompt chunk size (Sec. 3.3, Eq. 3) and its number of parallel-drafting
+ * steps (Sec. 3.5, Eq. 6).
+ *   g(.) is kept on a uniform grid of `num_bins` token sizes `bin_width` apart;
+ *   an observation updates the grid point nearest to the smoothed token size;
+ *   g is linear between observed points, continues with the outermost slope
+ *   beyond them, is constant with one observed point and 0 with none.  The
+ *   first observation of any moving average is taken as is.
+ * hat_ctrl_observe(mu_hat, eta_hat)       Eq. 1 then Eq. 2 (tokens, seconds)
+ * hat_ctrl_device_observe(i, gamma, beta_up, beta_down)   moving averages of device i's drafting delay per step
+ *                                         (seconds) and up/down bandwidths (bytes per second)
+ * hat_ctrl_chunk_size(i, A, P, x_min, x_max, &X)   smallest integer X in [x_min, x_max] with
+ *                                         X*A/beta_up >= (g(mu) + g(mu + X)) / P   (A = bytes of hidden state per
+ *                                         token, P = pipeline length); x_max if there is none
+ * hat_ctrl_parallel_draft_steps(i, n, A, &lambda)  floor((n*A/beta_up + g(mu) + n*A/beta_down) / gamma) for a draft
+ *                                         sequence of n tokens
+ * Errors: INVALID_ARG (null, out-of-range device, device never observed, non-positive rates, alpha outside [0,1]).
+ */
+typedef struct hat_ctrl hat_ctrl;
+int hat_ctrl_create(double alpha, double bin_width, int num_bins, int max_devices, hat_ctrl** out);
+int hat_ctrl_destroy(hat_ctrl* ctrl);   /* NULL is accepted */
+int hat_ctrl_observe(hat_ctrl* ctrl, double mu_hat, double eta_hat);
+int hat_ctrl_mu(const hat_ctrl* ctrl, double* out);
+int hat_ctrl_predict(const hat_ctrl* ctrl, double tokens, double* out);
+int hat_ctrl_device_observe(hat_ctrl* ctrl, int device, double gamma_hat, double beta_up_hat, double beta_down_hat);
+int hat_ctrl_device_state(const hat_ctrl* ctrl, int device, double* gamma, double* beta_up, double* beta_down);
+int hat_ctrl_chunk_size(const hat_ctrl* ctrl, int device, double bytes_per_token, int pipeline_length,
+                        int x_min, int x_max, int* out);
+int hat_ctrl_parallel_draft_steps(const hat_ctrl* ctrl, int device, int draft_len, double bytes_per_token, int* out);
+
+/*
  * Streaming attention for callers that must not allocate.  (The paper has no
  * counterpart: this is a deployment convenience of this library.)
  *

@@ -35,6 +35,8 @@ EXPORTS = [
     "hat_kv_append", "hat_chunk_attention", "hat_plan_staging_bytes", "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
     "hat_verify_attention_static", "hat_plan_set_wait_limit",
+    "hat_ctrl_create", "hat_ctrl_destroy", "hat_ctrl_observe", "hat_ctrl_mu", "hat_ctrl_predict",
+    "hat_ctrl_device_observe", "hat_ctrl_device_state", "hat_ctrl_chunk_size", "hat_ctrl_parallel_draft_steps",
 ]
 HAT_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 HAT_STATIC_SPLITS = 8
@@ -121,6 +123,16 @@ def lib() -> C.CDLL:
         L.hat_plan_read_timing.argtypes = [vp, vp, i32, C.POINTER(i32)]
         L.hat_plan_set_wait_limit.restype = i32
         L.hat_plan_set_wait_limit.argtypes = [vp, C.c_longlong, i32]
+        dbl = C.c_double
+        for name, args in (("hat_ctrl_create", [dbl, dbl, i32, i32, C.POINTER(vp)]), ("hat_ctrl_destroy", [vp]),
+                           ("hat_ctrl_observe", [vp, dbl, dbl]), ("hat_ctrl_mu", [vp, C.POINTER(dbl)]),
+                           ("hat_ctrl_predict", [vp, dbl, C.POINTER(dbl)]),
+                           ("hat_ctrl_device_observe", [vp, i32, dbl, dbl, dbl]),
+                           ("hat_ctrl_device_state", [vp, i32, C.POINTER(dbl), C.POINTER(dbl), C.POINTER(dbl)]),
+                           ("hat_ctrl_chunk_size", [vp, i32, dbl, i32, i32, i32, C.POINTER(i32)]),
+                           ("hat_ctrl_parallel_draft_steps", [vp, i32, i32, dbl, C.POINTER(i32)])):
+            getattr(L, name).restype = i32
+            getattr(L, name).argtypes = args
         L.hat_verify_attention_static.restype = i32
         L.hat_verify_attention_static.argtypes = [C.POINTER(hat_cache_desc), i32, i32, i32, i32, vp, vp, vp, vp,
                                                   vp, vp, vp, C.c_float, vp]
@@ -279,3 +291,65 @@ def hat_verify_attention_static(cache: hat_cache_desc, num_requests: int, num_q_
 def hat_plan_set_wait_limit(plan, cycles: int = 0, withhold_next_call: bool = False) -> None:
     _check(lib().hat_plan_set_wait_limit(_h(plan), int(cycles), 1 if withhold_next_call else 0),
            "hat_plan_set_wait_limit")
+
+
+class Ctrl:
+    """Owner of a hat_ctrl* (the cloud-side state monitor and chunk-size controller)."""
+
+    def __init__(self, alpha: float = 0.8, bin_width: float = 64.0, num_bins: int = 256, max_devices: int = 64):
+        h = C.c_void_p()
+        _check(lib().hat_ctrl_create(alpha, bin_width, num_bins, max_devices, C.byref(h)), "hat_ctrl_create")
+        self.handle = h.value
+
+    def close(self):
+        if self.handle:
+            lib().hat_ctrl_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def hat_ctrl_observe(ctrl: Ctrl, mu_hat: float, eta_hat: float) -> None:
+    _check(lib().hat_ctrl_observe(ctrl.handle, float(mu_hat), float(eta_hat)), "hat_ctrl_observe")
+
+
+def hat_ctrl_mu(ctrl: Ctrl) -> float:
+    v = C.c_double()
+    _check(lib().hat_ctrl_mu(ctrl.handle, C.byref(v)), "hat_ctrl_mu")
+    return v.value
+
+
+def hat_ctrl_predict(ctrl: Ctrl, tokens: float) -> float:
+    v = C.c_double()
+    _check(lib().hat_ctrl_predict(ctrl.handle, float(tokens), C.byref(v)), "hat_ctrl_predict")
+    return v.value
+
+
+def hat_ctrl_device_observe(ctrl: Ctrl, device: int, gamma: float, beta_up: float, beta_down: float) -> None:
+    _check(lib().hat_ctrl_device_observe(ctrl.handle, int(device), float(gamma), float(beta_up), float(beta_down)),
+           "hat_ctrl_device_observe")
+
+
+def hat_ctrl_device_state(ctrl: Ctrl, device: int):
+    g, u, d = C.c_double(), C.c_double(), C.c_double()
+    _check(lib().hat_ctrl_device_state(ctrl.handle, int(device), C.byref(g), C.byref(u), C.byref(d)),
+           "hat_ctrl_device_state")
+    return g.value, u.value, d.value
+
+
+def hat_ctrl_chunk_size(ctrl: Ctrl, device: int, bytes_per_token: float, pipeline_length: int, x_min: int, x_max: int) -> int:
+    v = C.c_int()
+    _check(lib().hat_ctrl_chunk_size(ctrl.handle, int(device), float(bytes_per_token), int(pipeline_length), int(x_min),
+                                     int(x_max), C.byref(v)), "hat_ctrl_chunk_size")
+    return v.value
+
+
+def hat_ctrl_parallel_draft_steps(ctrl: Ctrl, device: int, draft_len: int, bytes_per_token: float) -> int:
+    v = C.c_int()
+    _check(lib().hat_ctrl_parallel_draft_steps(ctrl.handle, int(device), int(draft_len), float(bytes_per_token),
+                                               C.byref(v)), "hat_ctrl_parallel_draft_steps")
+    return v.value
