@@ -207,10 +207,11 @@ int hat_chunk_attention_host(const hat_cache_desc* cache, const hat_plan* plan,
  * hat_plan_enable_timing, each of the next max_calls calls of
  * hat_chunk_attention / hat_chunk_attention_host on this plan records CUDA
  * events on its stream around each kernel it launches (this creates
- * 5*max_calls events once, here, not in the attention call).
+ * 8*max_calls events once, here, not in the attention call).
  * hat_plan_read_timing waits for the recorded events and writes, per recorded
  * call, HAT_TIMING_SLOTS durations in milliseconds: [0] KV append, [1] tile
- * (prefill-class) attention, [2] streaming (verify-class) attention, [3] merge;
+ * (prefill-class) attention, [2] streaming (verify-class) attention with the
+ * merge of its rows, [3] merge of tile-class rows;
  * 0 where a kernel was not launched.  It then rewinds the recorder.
  *   ms          host, [capacity_calls][HAT_TIMING_SLOTS]
  *   num_calls   host, out: calls written
@@ -218,6 +219,20 @@ int hat_chunk_attention_host(const hat_cache_desc* cache, const hat_plan* plan,
 #define HAT_TIMING_SLOTS 4
 int hat_plan_enable_timing(hat_plan* plan, int max_calls);
 int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num_calls);
+
+/*
+ * Decode-phase requests are not held back by prompt chunks (Sec. 2.1 "Batched
+ * Inference": long prefills delay the decode requests of the same batch; Sec.
+ * 3.3).  hat_chunk_attention computes the streaming-class chunks (draft
+ * verification, chunk_len <= 16) first and records an event owned by the plan
+ * as soon as their out/lse rows are final, before the tile kernel for the
+ * prompt chunks of the same batch starts.
+ *   hat_plan_verify_event   the cudaEvent_t (as void*), e.g. for cudaStreamWaitEvent on the caller's own stream
+ *                           that returns those rows to the devices; it is re-recorded by every attention call
+ *   hat_plan_wait_verify    blocks the host until the event of the latest call has occurred
+ */
+int hat_plan_verify_event(const hat_plan* plan, void** event_out);
+int hat_plan_wait_verify(const hat_plan* plan);
 
 /*
  * Read and clear the device-side status word of a plan (synchronises

@@ -35,6 +35,7 @@ EXPORTS = [
     "hat_kv_append", "hat_chunk_attention", "hat_plan_staging_bytes", "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
     "hat_verify_attention_static", "hat_plan_set_wait_limit",
+    "hat_plan_verify_event", "hat_plan_wait_verify",
     "hat_ctrl_create", "hat_ctrl_destroy", "hat_ctrl_observe", "hat_ctrl_mu", "hat_ctrl_predict",
     "hat_ctrl_device_observe", "hat_ctrl_device_state", "hat_ctrl_chunk_size", "hat_ctrl_parallel_draft_steps",
 ]
@@ -133,6 +134,10 @@ def lib() -> C.CDLL:
                            ("hat_ctrl_parallel_draft_steps", [vp, i32, i32, dbl, C.POINTER(i32)])):
             getattr(L, name).restype = i32
             getattr(L, name).argtypes = args
+        L.hat_plan_verify_event.restype = i32
+        L.hat_plan_verify_event.argtypes = [vp, C.POINTER(vp)]
+        L.hat_plan_wait_verify.restype = i32
+        L.hat_plan_wait_verify.argtypes = [vp]
         L.hat_verify_attention_static.restype = i32
         L.hat_verify_attention_static.argtypes = [C.POINTER(hat_cache_desc), i32, i32, i32, i32, vp, vp, vp, vp,
                                                   vp, vp, vp, C.c_float, vp]
@@ -353,3 +358,14 @@ def hat_ctrl_parallel_draft_steps(ctrl: Ctrl, device: int, draft_len: int, bytes
     _check(lib().hat_ctrl_parallel_draft_steps(ctrl.handle, int(device), int(draft_len), float(bytes_per_token),
                                                C.byref(v)), "hat_ctrl_parallel_draft_steps")
     return v.value
+
+
+def hat_plan_verify_event(plan) -> int:
+    """Raw cudaEvent_t recorded once the streaming-class rows of a call are final."""
+    ev = C.c_void_p()
+    _check(lib().hat_plan_verify_event(_h(plan), C.byref(ev)), "hat_plan_verify_event")
+    return ev.value
+
+
+def hat_plan_wait_verify(plan) -> None:
+    _check(lib().hat_plan_wait_verify(_h(plan)), "hat_plan_wait_verify")

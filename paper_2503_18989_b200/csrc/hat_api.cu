@@ -137,19 +137,23 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     if (psplit > 0) psplit = round_up(psplit, key_granule);
     info.prefill_split_len = psplit;
 
+    // streaming-class requests first: their merge rows form the head of merge_rows, so that they can be merged (and
+    // announced through the plan's event) before the tile kernel runs
     for (int r = 0; r < R; ++r) {
-        int C = p->chunk_len[r], P = p->prefix_len[r];
-        if (C <= 0) continue;
-        if (C <= verify_max_rows) {
-            int kv_end = P + C;
-            emit_tile(p, p->verify_items, r, 0, C, kv_end, split_len_for(kv_end, vsplit, kPageSize));
-        } else {
-            for (int row0 = 0; row0 < C; row0 += tile_rows) {
-                int rows_valid = std::min(tile_rows, C - row0);
-                int kv_end = P + row0 + rows_valid;
-                int sl = psplit > 0 ? split_len_for(kv_end, psplit, key_granule) : 0;
-                emit_tile(p, p->prefill_items, r, row0, rows_valid, kv_end, sl);
-            }
+        const int C = p->chunk_len[r], P = p->prefix_len[r];
+        if (C <= 0 || C > verify_max_rows) continue;
+        const int kv_end = P + C;
+        emit_tile(p, p->verify_items, r, 0, C, kv_end, split_len_for(kv_end, vsplit, kPageSize));
+    }
+    p->num_verify_merge_rows = (int)p->merge_rows.size();
+    for (int r = 0; r < R; ++r) {
+        const int C = p->chunk_len[r], P = p->prefix_len[r];
+        if (C <= verify_max_rows) continue;
+        for (int row0 = 0; row0 < C; row0 += tile_rows) {
+            const int rows_valid = std::min(tile_rows, C - row0);
+            const int kv_end = P + row0 + rows_valid;
+            const int sl = psplit > 0 ? split_len_for(kv_end, psplit, key_granule) : 0;
+            emit_tile(p, p->prefill_items, r, row0, rows_valid, kv_end, sl);
         }
     }
     // longest pieces first so the tail of the grid is made of short ones
@@ -308,6 +312,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->part_rows = 0;
     p->dev_blob = nullptr;
     p->timing = nullptr;
+    p->num_verify_merge_rows = 0;
+    p->ev_verify = nullptr;
     p->wait_cycles = 2000000000LL;
     p->withhold_next = 0;
     std::memset(&p->info, 0, sizeof p->info);
@@ -365,6 +371,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     if (!p->host_only) {
         st = upload(p);
         if (st != HAT_OK) { hat_plan_destroy(p); return st; }
+        cudaError_t ee = cudaEventCreateWithFlags(&p->ev_verify, cudaEventDisableTiming);
+        if (ee != cudaSuccess) { p->ev_verify = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
     }
     *out = p;
     return HAT_OK;
@@ -389,6 +397,7 @@ int hat_plan_destroy(hat_plan* plan) {
         for (cudaEvent_t ev : plan->timing->events) cudaEventDestroy(ev);
         delete plan->timing;
     }
+    if (plan->ev_verify) cudaEventDestroy(plan->ev_verify);
     if (plan->dev_blob) {
         cudaError_t e = cudaFree(plan->dev_blob);
         if (e != cudaSuccess) st = cuda_fail(e);
@@ -427,23 +436,20 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    // optional event recorder: slot boundaries 0..4 around append, tile, streaming, merge
+    // optional event recorder: a start and an end event per slot (append, tile, streaming, merge)
     Timing* tm = plan->timing;
     int call = -1;
     if (tm && tm->next < tm->max_calls) call = tm->next++;
-    auto mark = [&](int boundary) {
-        if (call >= 0) cudaEventRecord(tm->events[(size_t)call * 5 + boundary], s);
+    auto mark = [&](int slot, int end) {
+        if (call >= 0) cudaEventRecord(tm->events[((size_t)call * HAT_TIMING_SLOTS + slot) * 2 + end], s);
+        if (call >= 0 && end) tm->launched[(size_t)call * HAT_TIMING_SLOTS + slot] = 1;
     };
-    auto ran = [&](int slot) {
-        if (call >= 0) tm->launched[(size_t)call * HAT_TIMING_SLOTS + slot] = 1;
-    };
-    mark(0);
     if (k_new) {
+        mark(0, 0);
         e = launch_kv_append(plan, view_of(cache), cache->k_pool, cache->v_pool, k_new, v_new, s);
         if (e != cudaSuccess) return cuda_fail(e);
-        ran(0);
+        mark(0, 1);
     }
-    mark(1);
     AttnArgs a;
     a.plan = plan->dev;
     a.cache = view_of(cache);
@@ -459,27 +465,44 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
     a.withhold = plan->withhold_next;
     const_cast<hat_plan*>(plan)->withhold_next = 0;
 
+    // Decode-phase (draft verification) requests first: their rows are final, and announced through the plan's event,
+    // before the prompt chunks of the same batch are computed, so that they are not held back by them.
+    const int n_vm = plan->num_verify_merge_rows, n_m = (int)plan->merge_rows.size();
+    if (!plan->verify_items.empty()) {
+        mark(2, 0);
+        e = plan->info.stream_kernel == 1 ? launch_attn_stream(plan, a, s)
+                                          : launch_attn_mma(plan, a, /*verify_class=*/true, s);
+        if (e == cudaSuccess && n_vm > 0) e = launch_merge(plan, a, 0, n_vm, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        mark(2, 1);
+    }
+    if (plan->ev_verify && (e = cudaEventRecord(plan->ev_verify, s)) != cudaSuccess) return cuda_fail(e);
     if (!plan->prefill_items.empty()) {
+        mark(1, 0);
         e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
                                            : launch_attn_mma(plan, a, /*verify_class=*/false, s);
         if (e != cudaSuccess) return cuda_fail(e);
-        ran(1);
+        mark(1, 1);
     }
-    mark(2);
-    if (!plan->verify_items.empty()) {
-        e = plan->info.stream_kernel == 1 ? launch_attn_stream(plan, a, s)
-                                          : launch_attn_mma(plan, a, /*verify_class=*/true, s);
+    if (n_m > n_vm) {
+        mark(3, 0);
+        e = launch_merge(plan, a, n_vm, n_m - n_vm, s);
         if (e != cudaSuccess) return cuda_fail(e);
-        ran(2);
+        mark(3, 1);
     }
-    mark(3);
-    if (!plan->merge_rows.empty()) {
-        e = launch_merge(plan, a, s);
-        if (e != cudaSuccess) return cuda_fail(e);
-        ran(3);
-    }
-    mark(4);
     return HAT_OK;
+}
+
+int hat_plan_verify_event(const hat_plan* plan, void** event_out) {
+    if (!plan || !event_out || plan->host_only) return HAT_ERR_INVALID_ARG;
+    *event_out = plan->ev_verify;
+    return HAT_OK;
+}
+
+int hat_plan_wait_verify(const hat_plan* plan) {
+    if (!plan || plan->host_only || !plan->ev_verify) return HAT_ERR_INVALID_ARG;
+    cudaError_t e = cudaEventSynchronize(plan->ev_verify);
+    return e == cudaSuccess ? HAT_OK : cuda_fail(e);
 }
 
 int hat_plan_enable_timing(hat_plan* plan, int max_calls) {
@@ -491,7 +514,7 @@ int hat_plan_enable_timing(hat_plan* plan, int max_calls) {
     }
     Timing* tm = new (std::nothrow) Timing();
     if (!tm) return HAT_ERR_INVALID_ARG;
-    tm->events.resize((size_t)max_calls * 5);
+    tm->events.resize((size_t)max_calls * HAT_TIMING_SLOTS * 2);
     for (size_t i = 0; i < tm->events.size(); ++i) {
         cudaError_t e = cudaEventCreate(&tm->events[i]);
         if (e != cudaSuccess) {
@@ -511,12 +534,13 @@ int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num
     Timing* tm = plan->timing;
     const int n = std::min(tm->next, capacity_calls);
     for (int c = 0; c < n; ++c) {
-        cudaError_t e = cudaEventSynchronize(tm->events[(size_t)c * 5 + 4]);
-        if (e != cudaSuccess) return cuda_fail(e);
         for (int sl = 0; sl < HAT_TIMING_SLOTS; ++sl) {
             float t = 0.f;
             if (tm->launched[(size_t)c * HAT_TIMING_SLOTS + sl]) {
-                e = cudaEventElapsedTime(&t, tm->events[(size_t)c * 5 + sl], tm->events[(size_t)c * 5 + sl + 1]);
+                cudaEvent_t e0 = tm->events[((size_t)c * HAT_TIMING_SLOTS + sl) * 2];
+                cudaEvent_t e1 = tm->events[((size_t)c * HAT_TIMING_SLOTS + sl) * 2 + 1];
+                cudaError_t e = cudaEventSynchronize(e1);
+                if (e == cudaSuccess) e = cudaEventElapsedTime(&t, e0, e1);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
             ms[(size_t)c * HAT_TIMING_SLOTS + sl] = t;

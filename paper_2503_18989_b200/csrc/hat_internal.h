@@ -69,7 +69,7 @@ struct AttnArgs {
 }  // namespace hat
 
 namespace hat {
-// Event recorder for the optional per-kernel timing (5 events per recorded call).
+// Event recorder for the optional per-kernel timing (a start and an end event per slot and recorded call).
 struct Timing {
     std::vector<cudaEvent_t> events;
     std::vector<uint8_t> launched;   // [call][slot]
@@ -90,6 +90,8 @@ struct hat_plan {
     int64_t part_rows;          // partial rows in the workspace
     hat_plan_info info;
     hat::Timing* timing;        // null unless hat_plan_enable_timing was called
+    int num_verify_merge_rows;  // merge rows of streaming-class requests; they come first in merge_rows
+    cudaEvent_t ev_verify;      // recorded in every attention call once the streaming-class rows are final
     long long wait_cycles;      // bound of device-side waits (default: about a second)
     int withhold_next;          // self test of the bounded waits: applies to the next attention call only
     void* dev_blob;             // one allocation holding every device array
@@ -101,7 +103,7 @@ namespace hat {
 cudaError_t launch_kv_append(const hat_plan* plan, const CacheView& cache, void* k_pool, void* v_pool,
                              const void* k_new, const void* v_new, cudaStream_t stream);
 cudaError_t launch_attn_mma(const hat_plan* plan, const AttnArgs& args, bool verify_class, cudaStream_t stream);
-cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, int first_row, int num_rows, cudaStream_t stream);
 // tcgen05 tile kernel (head_dim 128): whether a TMA descriptor can be built for this pool layout, and the launcher
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                           int64_t stride_head);

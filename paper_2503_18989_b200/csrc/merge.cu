@@ -53,17 +53,17 @@ merge_kernel(const MergeRow* __restrict__ rows, int num_rows, int H,
     if (lane == 0) lse[(int64_t)mr.row * H + h] = sum > 0.f ? ms + logf(sum) : -INFINITY;
 }
 
-cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
-    const int n = (int)plan->merge_rows.size();
-    if (n == 0) return cudaSuccess;
+cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, int first_row, int num_rows, cudaStream_t stream) {
+    const int n = num_rows;
+    if (n <= 0) return cudaSuccess;
     const int H = plan->num_heads;
     const int64_t units = (int64_t)n * H;
     const unsigned blocks = (unsigned)((units + 3) / 4);
     if (plan->head_dim == 128)
-        merge_kernel<128><<<blocks, 128, 0, stream>>>(plan->dev.merge_rows, n, H, args.part_out, args.part_lse,
+        merge_kernel<128><<<blocks, 128, 0, stream>>>(plan->dev.merge_rows + first_row, n, H, args.part_out, args.part_lse,
                                                       args.out, args.lse);
     else
-        merge_kernel<64><<<blocks, 128, 0, stream>>>(plan->dev.merge_rows, n, H, args.part_out, args.part_lse,
+        merge_kernel<64><<<blocks, 128, 0, stream>>>(plan->dev.merge_rows + first_row, n, H, args.part_out, args.part_lse,
                                                      args.out, args.lse);
     count_launch();
     return cudaGetLastError();
