@@ -362,6 +362,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         // the accumulator still holds the previous unit: wait until its rows are in registers
                         ok = mbar_wait(&bars->o_free[qt], f_cnt[qt] & 1, bars, status);
                         ++f_cnt[qt];
+                        o_busy[qt] = false;
                         if (!ok) return;
                     }
                     ok = mbar_wait(&bars->p_ready[qt], p_cnt[qt] & 1, bars, status);
@@ -393,7 +394,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         if (ok && j + 1 < u.n_all) issue_s(1, j + 1);
                     }
                 }
-                o_busy[0] = u.n_q0 > 0;
+                // a unit in which a tile had no keys leaves that tile's earlier hand-over pending
+                if (u.n_q0 > 0) o_busy[0] = true;
                 if (u.nq == 2) o_busy[1] = true;
                 kt_base += u.n_all;
             }

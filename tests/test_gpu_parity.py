@@ -296,6 +296,23 @@ def test_long_prefill_request_is_cut_into_at_most_32_key_ranges(cuda_device):
     assert_parity(got[0][1][samples[:, 1], 0], wl, "long prefill lse")
 
 
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_key_ranges_that_only_the_second_query_tile_sees(cuda_device, dtype, monkeypatch):
+    """Ranges of 256 keys over 256-row units whose prefix is 128 past a multiple of 256: the last range of every
+    unit lies wholly behind the first query tile's last row, so that tile has no work in it while the second
+    one has; with 2 heads and 120 requests every CTA of the persistent kernel strings several such units
+    between ordinary ones."""
+    monkeypatch.setenv("HAT_PREFILL_SPLIT_LEN", "256")
+    prefix = [128 + 256 * (r % 4) for r in range(120)]
+    chunk = [256 if r % 5 else 200 for r in range(120)]
+    sc = _manual(dtype, 2, 128, prefix, chunk, 23)
+    from paper_2503_18989_b200 import runner
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert ds.info["prefill_kernel"] == 1 and ds.info["prefill_split_len"] == 256 and ds.info["max_splits"] == 5
+    _check_full(sc, cuda_device)
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_random_small_batches(cuda_device, seed):
     """Seeded random batches that mix every chunk class, odd prefixes, both types, both head sizes and both
