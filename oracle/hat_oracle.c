@@ -25,6 +25,20 @@
  *                               sequence verified in a single inference step
  *                               (Sec. 2.1 "Speculative Decoding"; Sec. 3.4).
  *   hat_oracle_chunk_attention  the same for every (row, head) of a batch.
+ *
+ *   Two extensions beyond the paper's own models, both optional:
+ *     grouped query heads   num_q_heads = G * num_heads: query head h reads the
+ *                           K/V head h / G (the paper's models have G = 1:
+ *                           32 and 40 attention heads, Sec. 4.1).
+ *     tree_mask             for a chunk of at most 16 rows, word t of tree_mask
+ *                           (one per packed row) replaces the causal rule
+ *                           INSIDE the chunk: row t sees chunk position c iff
+ *                           bit c is set; the cached prefix stays fully
+ *                           visible.  This is the token-tree verification of
+ *                           the U-Medusa comparison system (Sec. 4.1, tree
+ *                           size 8); HAT's own drafts are a linear sequence
+ *                           (Sec. 3.4), i.e. the causal rule.  Longer chunks
+ *                           are prompt chunks and stay causal.
  *   hat_oracle_merge            combination of attention results computed over
  *                               disjoint key sets (exact identity of softmax;
  *                               not in the paper, used by split-KV kernels).
@@ -42,6 +56,7 @@
 #include <string.h>
 
 enum { HAT_ORACLE_FP16 = 0, HAT_ORACLE_BF16 = 1 };
+enum { HAT_ORACLE_TREE_MAX_ROWS = 16 };
 
 /* IEEE 754 binary16 -> double, exact. */
 static double half_bits_to_double(uint16_t h)
@@ -129,58 +144,79 @@ void hat_oracle_kv_append(uint16_t *k_pool, uint16_t *v_pool,
  */
 static void attend_one(const uint16_t *k_pool, const uint16_t *v_pool, int dtype,
                        int64_t stride_page, int64_t stride_token, int64_t stride_head,
-                       int page_size, int num_heads, int head_dim,
-                       const int32_t *cu_chunk, const int32_t *prefix_len,
+                       int page_size, int num_heads, int num_q_heads, int head_dim,
+                       const int32_t *cu_chunk, const int32_t *prefix_len, const int32_t *chunk_len,
                        const int32_t *block_table, int max_pages,
-                       const uint16_t *q, double sm_scale,
+                       const uint16_t *q, const uint32_t *tree_mask, double sm_scale,
                        int r, int i, int h, int64_t j_begin, int64_t j_end,
                        double *out, double *lse)
 {
-    int64_t visible_end = (int64_t)prefix_len[r] + i + 1;      /* keys 0 .. prefix+i */
+    int64_t P = prefix_len[r];
+    int64_t visible_end = P + i + 1;                            /* causal: keys 0 .. prefix+i */
+    int use_tree = tree_mask != NULL && chunk_len[r] <= HAT_ORACLE_TREE_MAX_ROWS;
+    uint32_t bits = 0;
+    if (use_tree) {
+        bits = tree_mask[(int64_t)cu_chunk[r] + i];
+        visible_end = P + chunk_len[r];                         /* any chunk position may be named */
+    }
     if (j_begin < 0) j_begin = 0;
     if (j_end < 0 || j_end > visible_end) j_end = visible_end;
     int64_t n = j_end - j_begin;
     for (int c = 0; c < head_dim; ++c) out[c] = 0.0;
-    if (n <= 0) { *lse = -INFINITY; return; }
+    *lse = -INFINITY;
+    if (n <= 0) return;
 
-    const uint16_t *qrow = q + (((int64_t)cu_chunk[r] + i) * num_heads + h) * head_dim;
+    int group = num_q_heads / num_heads;                        /* query heads per K/V head */
+    int hk = h / group;
+    const uint16_t *qrow = q + (((int64_t)cu_chunk[r] + i) * num_q_heads + h) * head_dim;
     double *s = (double *)malloc((size_t)n * sizeof(double));
+    char *seen = (char *)malloc((size_t)n);
 
     double m = -INFINITY;
+    int64_t count = 0;
     for (int64_t j = j_begin; j < j_end; ++j) {
+        seen[j - j_begin] = (char)(!use_tree || j < P || ((bits >> (j - P)) & 1u));
+        if (!seen[j - j_begin]) continue;
         int64_t off = slot_offset(block_table, max_pages, page_size, stride_page,
-                                  stride_token, stride_head, r, j, h);
+                                  stride_token, stride_head, r, j, hk);
         double dot = 0.0;
         for (int c = 0; c < head_dim; ++c)
             dot += widen(qrow[c], dtype) * widen(k_pool[off + c], dtype);
         s[j - j_begin] = sm_scale * dot;
         if (s[j - j_begin] > m) m = s[j - j_begin];
+        ++count;
     }
-    double l = 0.0;
-    for (int64_t j = j_begin; j < j_end; ++j) {
-        int64_t off = slot_offset(block_table, max_pages, page_size, stride_page,
-                                  stride_token, stride_head, r, j, h);
-        double w = exp(s[j - j_begin] - m);
-        l += w;
-        for (int c = 0; c < head_dim; ++c)
-            out[c] += w * widen(v_pool[off + c], dtype);
+    if (count > 0) {
+        double l = 0.0;
+        for (int64_t j = j_begin; j < j_end; ++j) {
+            if (!seen[j - j_begin]) continue;
+            int64_t off = slot_offset(block_table, max_pages, page_size, stride_page,
+                                      stride_token, stride_head, r, j, hk);
+            double w = exp(s[j - j_begin] - m);
+            l += w;
+            for (int c = 0; c < head_dim; ++c)
+                out[c] += w * widen(v_pool[off + c], dtype);
+        }
+        for (int c = 0; c < head_dim; ++c) out[c] /= l;
+        *lse = m + log(l);
     }
-    for (int c = 0; c < head_dim; ++c) out[c] /= l;
-    *lse = m + log(l);
+    free(seen);
     free(s);
 }
 
 /*
  * Attention for a list of sampled rows.  sample[5*t + {0,1,2,3,4}] =
- * (request, row within chunk, head, j_begin, j_end); out is [num_samples,
- * head_dim], lse is [num_samples].
+ * (request, row within chunk, query head, j_begin, j_end); out is [num_samples,
+ * head_dim], lse is [num_samples].  q is [T, num_q_heads, head_dim]; tree_mask
+ * is NULL or [T].
  */
 void hat_oracle_attention_rows(const uint16_t *k_pool, const uint16_t *v_pool, int dtype,
                                int64_t stride_page, int64_t stride_token, int64_t stride_head,
-                               int page_size, int num_heads, int head_dim,
+                               int page_size, int num_heads, int num_q_heads, int head_dim,
                                const int32_t *cu_chunk, const int32_t *prefix_len,
+                               const int32_t *chunk_len,
                                const int32_t *block_table, int max_pages,
-                               const uint16_t *q, double sm_scale,
+                               const uint16_t *q, const uint32_t *tree_mask, double sm_scale,
                                int64_t num_samples, const int64_t *sample,
                                double *out, double *lse)
 {
@@ -188,37 +224,38 @@ void hat_oracle_attention_rows(const uint16_t *k_pool, const uint16_t *v_pool, i
     for (int64_t t = 0; t < num_samples; ++t) {
         const int64_t *sm = sample + 5 * t;
         attend_one(k_pool, v_pool, dtype, stride_page, stride_token, stride_head, page_size,
-                   num_heads, head_dim, cu_chunk, prefix_len, block_table, max_pages, q, sm_scale,
+                   num_heads, num_q_heads, head_dim, cu_chunk, prefix_len, chunk_len, block_table,
+                   max_pages, q, tree_mask, sm_scale,
                    (int)sm[0], (int)sm[1], (int)sm[2], sm[3], sm[4],
                    out + t * head_dim, lse + t);
     }
 }
 
 /*
- * Attention for every (row, head) of a batch.  out is [T, num_heads, head_dim],
- * lse is [T, num_heads], T = cu_chunk[num_requests].  The cache must already
- * hold the chunk's own K/V (append first, then attend).
+ * Attention for every (row, query head) of a batch.  out is [T, num_q_heads,
+ * head_dim], lse is [T, num_q_heads], T = cu_chunk[num_requests].  The cache
+ * must already hold the chunk's own K/V (append first, then attend).
  */
 void hat_oracle_chunk_attention(const uint16_t *k_pool, const uint16_t *v_pool, int dtype,
                                 int64_t stride_page, int64_t stride_token, int64_t stride_head,
-                                int page_size, int num_heads, int head_dim,
+                                int page_size, int num_heads, int num_q_heads, int head_dim,
                                 int num_requests, const int32_t *cu_chunk,
                                 const int32_t *prefix_len, const int32_t *chunk_len,
                                 const int32_t *block_table, int max_pages,
-                                const uint16_t *q, double sm_scale,
+                                const uint16_t *q, const uint32_t *tree_mask, double sm_scale,
                                 double *out, double *lse)
 {
     for (int r = 0; r < num_requests; ++r) {
-        int64_t units = (int64_t)chunk_len[r] * num_heads;
+        int64_t units = (int64_t)chunk_len[r] * num_q_heads;
 #pragma omp parallel for schedule(dynamic, 1)
         for (int64_t u = 0; u < units; ++u) {
-            int i = (int)(u / num_heads);
-            int h = (int)(u % num_heads);
+            int i = (int)(u / num_q_heads);
+            int h = (int)(u % num_q_heads);
             int64_t row = (int64_t)cu_chunk[r] + i;
             attend_one(k_pool, v_pool, dtype, stride_page, stride_token, stride_head, page_size,
-                       num_heads, head_dim, cu_chunk, prefix_len, block_table, max_pages, q,
-                       sm_scale, r, i, h, 0, -1,
-                       out + (row * num_heads + h) * head_dim, lse + row * num_heads + h);
+                       num_heads, num_q_heads, head_dim, cu_chunk, prefix_len, chunk_len,
+                       block_table, max_pages, q, tree_mask, sm_scale, r, i, h, 0, -1,
+                       out + (row * num_q_heads + h) * head_dim, lse + row * num_q_heads + h);
         }
     }
 }

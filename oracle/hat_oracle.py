@@ -46,11 +46,11 @@ def lib() -> C.CDLL:
         L.hat_oracle_kv_append.restype = None
         L.hat_oracle_kv_append.argtypes = [vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp, i32, vp, vp]
         L.hat_oracle_attention_rows.restype = None
-        L.hat_oracle_attention_rows.argtypes = [vp, vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, vp, i32,
-                                                vp, dbl, i64, vp, vp, vp]
+        L.hat_oracle_attention_rows.argtypes = [vp, vp, i32, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp, i32,
+                                                vp, vp, dbl, i64, vp, vp, vp]
         L.hat_oracle_chunk_attention.restype = None
-        L.hat_oracle_chunk_attention.argtypes = [vp, vp, i32, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp,
-                                                 vp, i32, vp, dbl, vp, vp]
+        L.hat_oracle_chunk_attention.argtypes = [vp, vp, i32, i64, i64, i64, i32, i32, i32, i32, i32, vp, vp, vp,
+                                                 vp, i32, vp, vp, dbl, vp, vp]
         L.hat_oracle_merge.restype = None
         L.hat_oracle_merge.argtypes = [i32, i32, vp, vp, vp, vp]
         L.hat_oracle_threads.restype = i32
@@ -87,9 +87,22 @@ def kv_append(cache, k_pool: np.ndarray, v_pool: np.ndarray, step) -> None:
                                len(pl), _p(cu), _p(pl), _p(cl), _p(bt), bt.shape[1], _p(kn), _p(vn))
 
 
+def _tree(step, T):
+    """The step's optional tree mask as a contiguous uint32 [T] array (kept alive by the caller), or None."""
+    tm = getattr(step, "tree_mask", None)
+    if tm is None:
+        return None
+    tm = _c(tm, np.uint32)
+    assert tm.shape == (T,)
+    return tm
+
+
 def chunk_attention(cache, k_pool, v_pool, step, sm_scale: float | None = None):
-    """(out [T,H,d] float64, lse [T,H] float64) for every row of the batch."""
-    H, d = cache.num_heads, cache.head_dim
+    """(out [T,Hq,d] float64, lse [T,Hq] float64) for every row of the batch; Hq = step.q.shape[1] query
+    heads over cache.num_heads K/V heads."""
+    Hkv, d = cache.num_heads, cache.head_dim
+    H = int(step.q.shape[1])
+    assert H % Hkv == 0
     if sm_scale is None:
         sm_scale = 1.0 / float(np.sqrt(np.float64(d)))
     cu, pl, cl = _c(step.cu_chunk, np.int32), _c(step.prefix_len, np.int32), _c(step.chunk_len, np.int32)
@@ -98,17 +111,20 @@ def chunk_attention(cache, k_pool, v_pool, step, sm_scale: float | None = None):
     T = int(cu[-1])
     out = np.zeros((T, H, d), dtype=np.float64)
     lse = np.zeros((T, H), dtype=np.float64)
+    tm = _tree(step, T)
     lib().hat_oracle_chunk_attention(_p(k_pool), _p(v_pool), DTYPE_CODE[cache.dtype], cache.stride_page,
-                                     cache.stride_token, cache.stride_head, cache.page_size, H, d,
+                                     cache.stride_token, cache.stride_head, cache.page_size, Hkv, H, d,
                                      len(pl), _p(cu), _p(pl), _p(cl), _p(bt), bt.shape[1], _p(q),
-                                     float(sm_scale), _p(out), _p(lse))
+                                     None if tm is None else _p(tm), float(sm_scale), _p(out), _p(lse))
     return out, lse
 
 
 def attention_rows(cache, k_pool, v_pool, step, samples, sm_scale: float | None = None):
     """Attention for sampled rows.  `samples` is an array [n, 3] of (request, row, head) or
-    [n, 5] of (request, row, head, j_begin, j_end).  Returns (out [n, d], lse [n])."""
-    H, d = cache.num_heads, cache.head_dim
+    [n, 5] of (request, row, query head, j_begin, j_end).  Returns (out [n, d], lse [n])."""
+    Hkv, d = cache.num_heads, cache.head_dim
+    H = int(step.q.shape[1])
+    assert H % Hkv == 0
     if sm_scale is None:
         sm_scale = 1.0 / float(np.sqrt(np.float64(d)))
     s = np.asarray(samples, dtype=np.int64)
@@ -117,14 +133,16 @@ def attention_rows(cache, k_pool, v_pool, step, samples, sm_scale: float | None 
     if s.shape[1] == 3:
         s = np.concatenate([s, np.zeros((len(s), 1), np.int64), -np.ones((len(s), 1), np.int64)], axis=1)
     s = np.ascontiguousarray(s)
-    cu, pl = _c(step.cu_chunk, np.int32), _c(step.prefix_len, np.int32)
+    cu, pl, cl = _c(step.cu_chunk, np.int32), _c(step.prefix_len, np.int32), _c(step.chunk_len, np.int32)
     bt = _c(step.block_table, np.int32)
     q = _c(step.q, np.uint16)
     out = np.zeros((len(s), d), dtype=np.float64)
     lse = np.zeros((len(s),), dtype=np.float64)
+    tm = _tree(step, int(cu[-1]))
     lib().hat_oracle_attention_rows(_p(k_pool), _p(v_pool), DTYPE_CODE[cache.dtype], cache.stride_page,
-                                    cache.stride_token, cache.stride_head, cache.page_size, H, d,
-                                    _p(cu), _p(pl), _p(bt), bt.shape[1], _p(q), float(sm_scale),
+                                    cache.stride_token, cache.stride_head, cache.page_size, Hkv, H, d,
+                                    _p(cu), _p(pl), _p(cl), _p(bt), bt.shape[1], _p(q),
+                                    None if tm is None else _p(tm), float(sm_scale),
                                     len(s), _p(s), _p(out), _p(lse))
     return out, lse
 

@@ -120,9 +120,10 @@ class Step:
     chunk_len: np.ndarray    # int32 [R]  rows sent up this step per request
     cu_chunk: np.ndarray     # int32 [R+1] exclusive prefix sum of chunk_len
     block_table: np.ndarray  # int32 [R, max_pages] physical page ids, -1 where unused
-    q: np.ndarray            # uint16 [T, H, d]
+    q: np.ndarray            # uint16 [T, Hq, d]   Hq = G * H query heads (G = 1 in the paper's models)
     k_new: np.ndarray        # uint16 [T, H, d]
     v_new: np.ndarray        # uint16 [T, H, d]
+    tree_mask: "np.ndarray | None" = None   # uint32 [T]: bit c = row sees chunk position c (chunks of <= 16 rows)
 
     @property
     def num_requests(self) -> int:
@@ -153,14 +154,15 @@ def _pages_for(tokens: int) -> int:
 
 def _make_step(rng_vals_seed: int, dtype: str, H: int, d: int,
                prefix_len: Sequence[int], chunk_len: Sequence[int],
-               block_table: np.ndarray) -> Step:
+               block_table: np.ndarray, q_heads: int | None = None) -> Step:
     prefix_len = np.asarray(prefix_len, dtype=np.int32)
     chunk_len = np.asarray(chunk_len, dtype=np.int32)
     cu = np.zeros(len(chunk_len) + 1, dtype=np.int32)
     np.cumsum(chunk_len, out=cu[1:])
     T = int(cu[-1])
     n = T * H * d
-    q = normal_bits(n, dtype, rng_vals_seed + 1).reshape(T, H, d)
+    Hq = H if q_heads is None else int(q_heads)
+    q = normal_bits(T * Hq * d, dtype, rng_vals_seed + 1).reshape(T, Hq, d)
     k = normal_bits(n, dtype, rng_vals_seed + 2).reshape(T, H, d)
     v = normal_bits(n, dtype, rng_vals_seed + 3).reshape(T, H, d)
     return Step(prefix_len, chunk_len, cu, np.ascontiguousarray(block_table, dtype=np.int32), q, k, v)
@@ -234,16 +236,42 @@ def ragged_prefill(num_requests: int = 30, max_prefix: int = 4096,
                      "ragged prefill batch, append in the same call")
 
 
+TREE_MAX_ROWS = 16
+
+
+def random_tree_masks(seed: int, chunk_len: Sequence[int]) -> np.ndarray:
+    """One uint32 word per packed row.  For a chunk of at most TREE_MAX_ROWS rows the rows form a random token
+    tree in topological order: node c hangs under a node drawn uniformly from {root, 0..c-1} and its word has
+    bit c and its parent's bits set (a row sees its ancestors and itself; the root is the cached prefix, which is
+    always visible).  Rows of longer chunks get the causal word (it is not consulted for them)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    words = []
+    for C in np.asarray(chunk_len, dtype=np.int64):
+        C = int(C)
+        if C > TREE_MAX_ROWS:
+            words.extend([0xFFFFFFFF] * C)
+            continue
+        mask = []
+        for c in range(C):
+            parent = int(rng.integers(-1, c))          # -1: hangs directly under the prefix
+            mask.append((mask[parent] if parent >= 0 else 0) | (1 << c))
+        words.extend(mask)
+    return np.asarray(words, dtype=np.uint32)
+
+
 def spec_verify(num_requests: int = 30, min_prefix: int = 512, max_prefix: int = 4096,
                 max_draft: int = 8, H: int = 32, d: int = 128, dtype: str = "fp16",
-                seed: int = SEED_BASE + 4) -> Scenario:
+                seed: int = SEED_BASE + 4, q_group: int = 1, tree: bool = False) -> Scenario:
     """Draft-verification batch: prefix uniform in [min_prefix, max_prefix] (any value, so
-    appends start mid-page), draft length uniform in [1, max_draft]."""
+    appends start mid-page), draft length uniform in [1, max_draft].  q_group > 1 gives q_group query
+    heads per K/V head; tree=True replaces the linear drafts by random token trees."""
     rng = np.random.Generator(np.random.PCG64(seed))
     prefix = rng.integers(min_prefix, max_prefix + 1, size=num_requests)
     chunk = rng.integers(1, max_draft + 1, size=num_requests)
     table, num_pages = _place_pages(rng, prefix + chunk, slack_pages=max(8, num_requests))
-    step = _make_step(seed + 100, dtype, H, d, prefix, chunk, table)
+    step = _make_step(seed + 100, dtype, H, d, prefix, chunk, table, q_heads=H * q_group)
+    if tree:
+        step.tree_mask = random_tree_masks(seed + 200, chunk)
     return _scenario("spec_verify", dtype, H, d, "paged", num_pages, [step], seed + 100,
                      "speculative verification batch")
 
@@ -251,9 +279,9 @@ def spec_verify(num_requests: int = 30, min_prefix: int = 512, max_prefix: int =
 def mixed_13b(num_prefill: int = 8, prefill_chunk: int = 512, max_prefill_prefix: int = 8192,
               num_verify: int = 32, draft: int = 4, min_verify_prefix: int = 1024,
               max_verify_prefix: int = 8192, H: int = 40, d: int = 128, dtype: str = "bf16",
-              seed: int = SEED_BASE + 5) -> Scenario:
+              seed: int = SEED_BASE + 5, q_group: int = 1, tree: bool = False) -> Scenario:
     """13B-shaped mixed batch: prefill chunks and verify chunks interleaved in one call
-    over one paged pool."""
+    over one paged pool.  q_group and tree as in spec_verify."""
     rng = np.random.Generator(np.random.PCG64(seed))
     p_pre = rng.integers(0, max_prefill_prefix + 1, size=num_prefill)
     p_ver = rng.integers(min_verify_prefix, max_verify_prefix + 1, size=num_verify)
@@ -262,7 +290,9 @@ def mixed_13b(num_prefill: int = 8, prefill_chunk: int = 512, max_prefill_prefix
     order = rng.permutation(len(prefix))          # devices arrive in no particular order
     prefix, chunk = prefix[order], chunk[order]
     table, num_pages = _place_pages(rng, prefix + chunk, slack_pages=max(8, len(prefix)))
-    step = _make_step(seed + 100, dtype, H, d, prefix, chunk, table)
+    step = _make_step(seed + 100, dtype, H, d, prefix, chunk, table, q_heads=H * q_group)
+    if tree:
+        step.tree_mask = random_tree_masks(seed + 200, chunk)
     return _scenario("mixed_13b", dtype, H, d, "paged", num_pages, [step], seed + 100,
                      "13B-shaped mixed prefill + verify batch")
 

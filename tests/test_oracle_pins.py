@@ -120,15 +120,24 @@ def test_constant_values_and_dominant_key():
 # brute force in pure Python (independent indexing, three passes, fsum)
 # ----------------------------------------------------------------------------
 def _brute_row(cache, k_pool, v_pool, st, r, i, h):
+    """h is the query head; with grouped query heads it reads K/V head h // G.  A tree mask, if the step has
+    one and the chunk is short, picks the visible chunk positions."""
     d = cache.head_dim
     kf = W.bits_to_f64(k_pool, cache.dtype); vf = W.bits_to_f64(v_pool, cache.dtype)
     qf = W.bits_to_f64(st.q, cache.dtype)
     row = int(st.cu_chunk[r]) + i
+    hk = h // (st.q.shape[1] // cache.num_heads)
+    P, Cn = int(st.prefix_len[r]), int(st.chunk_len[r])
+    tm = getattr(st, "tree_mask", None)
+    if tm is not None and Cn <= 16:
+        visible = list(range(P)) + [P + c for c in range(Cn) if (int(tm[row]) >> c) & 1]
+    else:
+        visible = list(range(P + i + 1))
     scores = []
     addr = []
-    for j in range(int(st.prefix_len[r]) + i + 1):
+    for j in visible:
         page = int(st.block_table[r][j // cache.page_size])
-        a = page * cache.stride_page + (j % cache.page_size) * cache.stride_token + h * cache.stride_head
+        a = page * cache.stride_page + (j % cache.page_size) * cache.stride_token + hk * cache.stride_head
         addr.append(a)
         scores.append(math.fsum(float(qf[row, h, c]) * float(kf[a + c]) for c in range(d)) / math.sqrt(d))
     top = max(scores)
@@ -164,6 +173,80 @@ def test_brute_force_rows(maker, kw):
     assert np.array_equal(so[0], out[int(st.cu_chunk[0]), 1])
     assert np.array_equal(so[1], out[int(st.cu_chunk[3]) - 1, 0])
     assert sl[0] == lse[int(st.cu_chunk[0]), 1]
+
+
+# ----------------------------------------------------------------------------
+# grouped query heads and token trees (extensions; the paper's models have one K/V head per query head, Sec. 4.1,
+# and HAT's own drafts are linear, Sec. 3.4; trees are the U-Medusa comparison system's, Sec. 4.1)
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("group,tree", [(4, False), (1, True), (2, True)])
+def test_brute_force_rows_grouped_heads_and_trees(group, tree):
+    sc = W.mixed_13b(num_prefill=1, prefill_chunk=20, max_prefill_prefix=40, num_verify=3, draft=7,
+                     min_verify_prefix=0, max_verify_prefix=50, H=2, d=64, seed=16, q_group=group, tree=tree)
+    cache, st = sc.cache, sc.steps[0]
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(cache, kp, vp, st)
+    out, lse = O.chunk_attention(cache, kp, vp, st)
+    assert out.shape == (st.total_rows, 2 * group, 64)
+    for r in range(st.num_requests):
+        for i in range(0, int(st.chunk_len[r]), 3):
+            for h in range(2 * group):
+                wo, wl = _brute_row(cache, kp, vp, st, r, i, h)
+                row = int(st.cu_chunk[r]) + i
+                assert np.allclose(out[row, h], wo, rtol=0, atol=1e-12)
+                assert lse[row, h] == pytest.approx(wl, abs=1e-12)
+
+
+def test_grouped_heads_equal_repeated_kv_heads():
+    """G query heads per K/V head == ordinary attention over a cache whose heads are each repeated G times."""
+    G, H, d = 3, 2, 64
+    sc = W.spec_verify(num_requests=3, min_prefix=5, max_prefix=60, max_draft=6, H=H, d=d, seed=17, q_group=G)
+    cache, st = sc.cache, sc.steps[0]
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(cache, kp, vp, st)
+    out, lse = O.chunk_attention(cache, kp, vp, st)
+    wide = W.CacheSpec(cache.dtype, H * G, d, cache.num_pages, "paged")
+    def widen_pool(pool):
+        x = pool.reshape(cache.num_pages, H, cache.page_size, d)
+        return np.ascontiguousarray(np.repeat(x, G, axis=1)).ravel()
+    out2, lse2 = O.chunk_attention(wide, widen_pool(kp), widen_pool(vp), st)
+    assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def test_causal_tree_mask_is_the_default_and_a_path_is_a_linear_draft():
+    sc = W.spec_verify(num_requests=4, min_prefix=0, max_prefix=40, max_draft=8, H=2, d=64, seed=18)
+    cache, st = sc.cache, sc.steps[0]
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(cache, kp, vp, st)
+    out, lse = O.chunk_attention(cache, kp, vp, st)
+    # (1) the lower-triangular words reproduce the causal rule bit for bit
+    st.tree_mask = np.concatenate([[(2 << i) - 1 for i in range(int(c))] for c in st.chunk_len]).astype(np.uint32)
+    out_t, lse_t = O.chunk_attention(cache, kp, vp, st)
+    assert np.array_equal(out, out_t) and np.array_equal(lse, lse_t)
+    # (2) a random tree: every node's row equals the last row of the LINEAR draft made of its root-to-node path
+    st.tree_mask = W.random_tree_masks(5, st.chunk_len)
+    out_t, lse_t = O.chunk_attention(cache, kp, vp, st)
+    kn = st.k_new.reshape(st.total_rows, -1); vn = st.v_new.reshape(st.total_rows, -1)
+    for r in range(st.num_requests):
+        P, Cn, base = int(st.prefix_len[r]), int(st.chunk_len[r]), int(st.cu_chunk[r])
+        for i in range(Cn):
+            path = [c for c in range(Cn) if (int(st.tree_mask[base + i]) >> c) & 1]
+            assert path[-1] == i
+            rows = [base + c for c in path]
+            lin = types.SimpleNamespace(prefix_len=np.asarray([P], np.int32), chunk_len=np.asarray([len(path)], np.int32),
+                                        cu_chunk=np.asarray([0, len(path)], np.int32),
+                                        block_table=st.block_table[r:r + 1], q=st.q[rows], k_new=st.k_new[rows],
+                                        v_new=st.v_new[rows])
+            kp2, vp2 = kp.copy(), vp.copy()
+            O.kv_append(cache, kp2, vp2, lin)          # the path's K/V at positions P .. P+len-1
+            out_l, lse_l = O.chunk_attention(cache, kp2, vp2, lin)
+            assert np.allclose(out_t[base + i], out_l[-1], rtol=0, atol=1e-13)
+            assert np.allclose(lse_t[base + i], lse_l[-1], rtol=0, atol=1e-13)
+    # (3) a word without any chunk bit at an empty prefix sees nothing
+    st0 = _step([0], [2], st.block_table[:1], st.q[:2], st.k_new[:2], st.v_new[:2])
+    st0.tree_mask = np.asarray([0, 2], np.uint32)
+    o0, l0 = O.chunk_attention(cache, kp, vp, st0)
+    assert np.all(o0[0] == 0) and np.all(l0[0] == -np.inf) and np.all(np.isfinite(l0[1]))
 
 
 # ----------------------------------------------------------------------------
