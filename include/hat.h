@@ -71,7 +71,7 @@ typedef struct hat_cache_desc {
     int32_t dtype;         /* HAT_DTYPE_FP16 | HAT_DTYPE_BF16 (q, k_new, v_new use the same type) */
     int32_t num_pages;     /* pages in each pool */
     int32_t page_size;     /* tokens per page; 16 is the only size built */
-    int32_t num_kv_heads;  /* must equal num_q_heads (multi-head attention) */
+    int32_t num_kv_heads;  /* K/V heads; num_q_heads must be a multiple of it (equal in the paper's models, Sec. 4.1) */
     int32_t head_dim;      /* 64 or 128 */
     int32_t reserved;      /* 0 */
     int64_t stride_page;
@@ -90,6 +90,15 @@ typedef struct hat_cache_desc {
  *   chunk_len   [num_requests]    rows of this chunk (>=0; 0 is a valid no-op)
  *   block_table [num_requests][max_pages] physical page ids; entries at or beyond
  *                                 ceil((prefix_len+chunk_len)/page_size) are ignored
+ * Two optional extensions (the paper's models and HAT's own drafts need neither):
+ *   num_q_heads = G * num_kv_heads   grouped query heads: query head h reads K/V head h / G; q, out and lse have
+ *                                 num_q_heads heads, k_new, v_new and the pools num_kv_heads
+ *   tree_mask   [T] or NULL       token-tree verification (the U-Medusa comparison system of Sec. 4.1; HAT's
+ *                                 drafts are a linear sequence, Sec. 3.4 = NULL).  For a request with
+ *                                 chunk_len <= 16, packed row t sees the whole cached prefix and chunk position c
+ *                                 iff bit c of tree_mask[t] is set (bits at or above chunk_len are ignored; a row
+ *                                 that sees nothing gets out = 0, lse = -inf).  Rows of longer chunks are prompt
+ *                                 chunks: causal, their words are not read.
  */
 typedef struct hat_batch_desc {
     int32_t        num_requests;
@@ -100,6 +109,7 @@ typedef struct hat_batch_desc {
     const int32_t* prefix_len;
     const int32_t* chunk_len;
     const int32_t* block_table;
+    const uint32_t* tree_mask;
 } hat_batch_desc;
 
 typedef struct hat_plan hat_plan;
@@ -119,8 +129,8 @@ typedef struct hat_plan_info {
     int32_t prefill_tile_rows;   /* query rows per CTA of the tile kernel */
     int32_t prefill_kernel;      /* 0 = mma.sync tile kernel, 1 = tcgen05 tile kernel */
     int64_t workspace_bytes;
-    int64_t attn_flops;          /* 4*d*H*sum_r [C_r*P_r + C_r*(C_r+1)/2] */
-    int64_t kv_read_bytes;       /* 2*sum_r (P_r+C_r)*H*d*elem: every visible K and V row read once per head */
+    int64_t attn_flops;          /* 4*d*H_q*sum_r [C_r*P_r + C_r*(C_r+1)/2] (causal count, also when a tree mask is given) */
+    int64_t kv_read_bytes;       /* 2*sum_r (P_r+C_r)*H_kv*d*elem: every visible K and V row read once per K/V head */
     int32_t stream_kernel;       /* 0 = cp.async streaming kernel, 1 = TMA streaming kernel */
     int32_t reserved;
 } hat_plan_info;

@@ -54,7 +54,7 @@ class hat_cache_desc(C.Structure):
 class hat_batch_desc(C.Structure):
     _fields_ = [("num_requests", C.c_int32), ("num_q_heads", C.c_int32), ("max_pages", C.c_int32),
                 ("flags", C.c_uint32), ("cu_chunk", C.c_void_p), ("prefix_len", C.c_void_p),
-                ("chunk_len", C.c_void_p), ("block_table", C.c_void_p)]
+                ("chunk_len", C.c_void_p), ("block_table", C.c_void_p), ("tree_mask", C.c_void_p)]
 
 
 class hat_plan_info(C.Structure):
@@ -208,16 +208,18 @@ def _h(plan) -> Optional[int]:
 
 
 def hat_plan_create(cache: hat_cache_desc, num_q_heads: int, cu_chunk, prefix_len, chunk_len, block_table,
-                    flags: int = 0) -> Plan:
-    """The four arrays are host int32 arrays (numpy); block_table is [num_requests, max_pages]."""
+                    flags: int = 0, tree_mask=None) -> Plan:
+    """The four arrays are host int32 arrays (numpy); block_table is [num_requests, max_pages]; tree_mask is
+    None or a host uint32 array with one word per packed row."""
     cu = np.ascontiguousarray(cu_chunk, dtype=np.int32)
     pl = np.ascontiguousarray(prefix_len, dtype=np.int32)
     cl = np.ascontiguousarray(chunk_len, dtype=np.int32)
     bt = np.ascontiguousarray(block_table, dtype=np.int32)
     R = int(pl.shape[0])
     max_pages = int(bt.shape[1]) if bt.ndim == 2 else 0
+    tm = None if tree_mask is None else np.ascontiguousarray(tree_mask, dtype=np.uint32)
     batch = hat_batch_desc(R, int(num_q_heads), max_pages, int(flags), _ptr(cu), _ptr(pl), _ptr(cl),
-                           _ptr(bt) if bt.size else None)
+                           _ptr(bt) if bt.size else None, None if tm is None or not tm.size else _ptr(tm))
     out = C.c_void_p()
     _check(lib().hat_plan_create(C.byref(cache), C.byref(batch), C.byref(out)), "hat_plan_create")
     return Plan(out.value, None)

@@ -125,7 +125,7 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
 
     const T* __restrict__ kpool = static_cast<const T*>(a.cache.k_pool);
     const T* __restrict__ vpool = static_cast<const T*>(a.cache.v_pool);
-    const int64_t head_off = (int64_t)h * a.cache.stride_head;
+    const int64_t head_off = (int64_t)(h / a.plan.group) * a.cache.stride_head;   // query head h reads K/V head h / G
 
     // ---- stage loader for this key group: tile index ti -> keys [kv_begin + ti*KB, +KB)
     const uint32_t stage_base = smem_base + Q_BYTES + kg * (STAGES * 2 * TILE_BYTES);
@@ -186,7 +186,15 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g+8 (log2 domain)
     const int lim0 = P + item.row0 + wm * 16 + g;                // last visible key of row g
     const int lim1 = lim0 + 8;
-    const int warp_last_visible = P + item.row0 + wm * 16 + 15;
+    // token tree (short chunks only): the words say which chunk positions rows g and g+8 see
+    const bool tree = a.plan.tree_mask != nullptr && C <= 16;
+    uint32_t bits0 = 0, bits1 = 0;
+    if (tree) {
+        const int i0 = item.row0 + wm * 16 + g;
+        if (i0 < C) bits0 = __ldg(a.plan.tree_mask + row_base + i0);
+        if (i0 + 8 < C) bits1 = __ldg(a.plan.tree_mask + row_base + i0 + 8);
+    }
+    const int warp_last_visible = tree ? P + C - 1 : P + item.row0 + wm * 16 + 15;
 
     for (int it = 0; it < n_my; ++it) {
         cp_async_wait<STAGES - 2>();
@@ -224,10 +232,16 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
 #pragma unroll
         for (int n = 0; n < KB / 8; ++n) {
             const int j = kb + n * 8 + 2 * t4;
-            s[n][0] = (j <= lim0 && j < kend) ? s[n][0] * a.scale_log2 : -INFINITY;
-            s[n][1] = (j + 1 <= lim0 && j + 1 < kend) ? s[n][1] * a.scale_log2 : -INFINITY;
-            s[n][2] = (j <= lim1 && j < kend) ? s[n][2] * a.scale_log2 : -INFINITY;
-            s[n][3] = (j + 1 <= lim1 && j + 1 < kend) ? s[n][3] * a.scale_log2 : -INFINITY;
+            bool a0 = j <= lim0, a1 = j + 1 <= lim0, b0 = j <= lim1, b1 = j + 1 <= lim1;
+            if (tree) {
+                const uint32_t sh0 = (uint32_t)min(max(j - P, 0), 31), sh1 = (uint32_t)min(max(j + 1 - P, 0), 31);
+                a0 = j < P || ((bits0 >> sh0) & 1u); a1 = j + 1 < P || ((bits0 >> sh1) & 1u);
+                b0 = j < P || ((bits1 >> sh0) & 1u); b1 = j + 1 < P || ((bits1 >> sh1) & 1u);
+            }
+            s[n][0] = (a0 && j < kend) ? s[n][0] * a.scale_log2 : -INFINITY;
+            s[n][1] = (a1 && j + 1 < kend) ? s[n][1] * a.scale_log2 : -INFINITY;
+            s[n][2] = (b0 && j < kend) ? s[n][2] * a.scale_log2 : -INFINITY;
+            s[n][3] = (b1 && j + 1 < kend) ? s[n][3] * a.scale_log2 : -INFINITY;
             mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
             mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
         }

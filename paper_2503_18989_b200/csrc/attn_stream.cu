@@ -75,7 +75,7 @@ __device__ __forceinline__ uint32_t q_off(int row, int c) { return (uint32_t)(ro
 
 template <bool BF16, int D>
 __global__ void __launch_bounds__(kWarps * 32)
-attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_constant__ CUtensorMap map_k,
+attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, int n_sub, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v) {
     using T = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
     constexpr int CH = D / 8, ON = D / 8, HALVES = D / 64;
@@ -88,12 +88,15 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Q_BYTES + kWarps * kSlots * SLOT_BYTES);
     const uint32_t sbase = s_u32(smem);
 
+    // A CTA serves one K/V head and 16 of the request's (chunk row i, query head gq of the head's group) pairs:
+    // MMA row m of slab `sub` is pair number sub * 16 + m = i * G + gq, so K/V are read once for the whole group.
     const WorkItem item = items[blockIdx.y];
-    const int h = blockIdx.x;
-    const int H = a.plan.num_heads;
+    const int h = blockIdx.x / n_sub, sub = blockIdx.x % n_sub;
+    const int H = a.plan.num_heads, G = a.plan.group;
     const int r = item.req;
     const int P = a.plan.prefix_len[r];
     const int C = a.plan.chunk_len[r];
+    if (sub * 16 >= C * G) return;                            // this request has fewer pairs
     const int row_base = a.plan.cu_chunk[r];
     const int32_t* __restrict__ table = a.plan.block_table + (int64_t)r * a.plan.max_pages;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
@@ -109,8 +112,9 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_
         for (int idx = tid; idx < 16 * CH; idx += kWarps * 32) {
             const int row = idx / CH, c = idx % CH;
             uint4 v = make_uint4(0, 0, 0, 0);
-            if (item.row0 + row < C)
-                v = __ldg(reinterpret_cast<const uint4*>(q + ((int64_t)(row_base + item.row0 + row) * H + h) * D) + c);
+            const int pair = sub * 16 + row, i = pair / G;
+            if (i < C)
+                v = __ldg(reinterpret_cast<const uint4*>(q + ((int64_t)(row_base + i) * H + h * G + pair % G) * D) + c);
             *reinterpret_cast<uint4*>(smem + q_off<D>(row, c)) = v;
         }
     }
@@ -154,7 +158,14 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_
 #pragma unroll
     for (int n = 0; n < ON; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // reference maxima (log2 units) and row sums, rows g and g+8
-    const int lim0 = P + item.row0 + g, lim1 = lim0 + 8;        // last visible key of rows g and g+8
+    // chunk rows of MMA rows g and g+8, and the chunk positions each may see: bit c <=> key P + c.  The causal rule
+    // (Sec. 2.1 / 3.4: a linear draft sequence) is bits 0..i; a token tree supplies its own words
+    const int i0 = (sub * 16 + g) / G, i1 = (sub * 16 + g + 8) / G;
+    uint32_t bits0 = i0 < C ? (2u << i0) - 1u : 0u, bits1 = i1 < C ? (2u << i1) - 1u : 0u;
+    if (a.plan.tree_mask != nullptr) {
+        if (i0 < C) bits0 = __ldg(a.plan.tree_mask + row_base + i0);
+        if (i1 < C) bits1 = __ldg(a.plan.tree_mask + row_base + i1);
+    }
     const int kend = item.kv_end;
     bool ok = true;
 
@@ -198,14 +209,21 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_
             mma16816<BF16>(s[1], qf[ks], b[2], b[3]);
         }
         float mx0 = -INFINITY, mx1 = -INFINITY;
-        if (kb + kPageSize - 1 > min(lim0, kend - 1)) {          // some key of the page is invisible to some row
+        if (kb + kPageSize > min(P, kend)) {                     // the page holds chunk positions or ends the range
 #pragma unroll
             for (int n = 0; n < 2; ++n) {
                 const int j = kb + n * 8 + 2 * t4;
-                s[n][0] = (j <= lim0 && j < kend) ? s[n][0] * a.scale_log2 : -INFINITY;
-                s[n][1] = (j + 1 <= lim0 && j + 1 < kend) ? s[n][1] * a.scale_log2 : -INFINITY;
-                s[n][2] = (j <= lim1 && j < kend) ? s[n][2] * a.scale_log2 : -INFINITY;
-                s[n][3] = (j + 1 <= lim1 && j + 1 < kend) ? s[n][3] * a.scale_log2 : -INFINITY;
+                // key j of the range: everything below P, bit j - P from there on (j < kend <= P + 16 bounds the shift)
+                const bool in0 = j < kend, in1 = j + 1 < kend;
+                const uint32_t sh0 = (uint32_t)min(max(j - P, 0), 31), sh1 = (uint32_t)min(max(j + 1 - P, 0), 31);
+                const bool a0 = in0 && (j < P || ((bits0 >> sh0) & 1u));
+                const bool a1 = in1 && (j + 1 < P || ((bits0 >> sh1) & 1u));
+                const bool b0 = in0 && (j < P || ((bits1 >> sh0) & 1u));
+                const bool b1 = in1 && (j + 1 < P || ((bits1 >> sh1) & 1u));
+                s[n][0] = a0 ? s[n][0] * a.scale_log2 : -INFINITY;
+                s[n][1] = a1 ? s[n][1] * a.scale_log2 : -INFINITY;
+                s[n][2] = b0 ? s[n][2] * a.scale_log2 : -INFINITY;
+                s[n][3] = b1 ? s[n][3] * a.scale_log2 : -INFINITY;
             }
         } else {
 #pragma unroll
@@ -327,21 +345,21 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, const __grid_
     constexpr float kLn2 = 0.6931471805599453f;
     const float lse0 = l0 > 0.f ? (mt0 + log2f(l0)) * kLn2 : -INFINITY;
     const float lse1 = l1 > 0.f ? (mt1 + log2f(l1)) * kLn2 : -INFINITY;
-    const int i0 = item.row0 + g, i1 = i0 + 8;
+    const int hq0 = h * G + (sub * 16 + g) % G, hq1 = h * G + (sub * 16 + g + 8) % G;
     float* obase; float* lbase; int64_t r0, r1;
     if (item.part < 0) { obase = a.out; lbase = a.lse; r0 = row_base + i0; r1 = row_base + i1; }
-    else { obase = a.part_out; lbase = a.part_lse; r0 = item.part + g; r1 = item.part + g + 8; }
+    else { obase = a.part_out; lbase = a.part_lse; r0 = item.part + i0; r1 = item.part + i1; }
     if (i0 < C) {
-        float* dst = obase + (r0 * H + h) * D + 2 * t4;
+        float* dst = obase + (r0 * H + hq0) * D + 2 * t4;
 #pragma unroll
         for (int n = 0; n < ON; ++n) *reinterpret_cast<float2*>(dst + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
-        if (t4 == 0) lbase[r0 * H + h] = lse0;
+        if (t4 == 0) lbase[r0 * H + hq0] = lse0;
     }
     if (i1 < C) {
-        float* dst = obase + (r1 * H + h) * D + 2 * t4;
+        float* dst = obase + (r1 * H + hq1) * D + 2 * t4;
 #pragma unroll
         for (int n = 0; n < ON; ++n) *reinterpret_cast<float2*>(dst + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
-        if (t4 == 0) lbase[r1 * H + h] = lse1;
+        if (t4 == 0) lbase[r1 * H + hq1] = lse1;
     }
 }
 
@@ -352,8 +370,8 @@ cudaError_t launch_one(const hat_plan* plan, const AttnArgs& args, const CUtenso
     auto kern = attn_stream_kernel<BF16, D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    kern<<<dim3(plan->num_heads, (unsigned)plan->verify_items.size()), kWarps * 32, smem, stream>>>(
-        args, plan->dev.verify_items, mk, mv);
+    kern<<<dim3(plan->num_kv_heads * plan->verify_subtiles, (unsigned)plan->verify_items.size()), kWarps * 32, smem, stream>>>(
+        args, plan->dev.verify_items, plan->verify_subtiles, mk, mv);
     count_launch();
     return cudaGetLastError();
 }
@@ -371,9 +389,9 @@ bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int6
 cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     CUtensorMap mk, mv;
-    if (!tma_encode_pool_map(&mk, bf16, args.cache.k_pool, plan->head_dim, plan->num_pages, plan->num_heads,
+    if (!tma_encode_pool_map(&mk, bf16, args.cache.k_pool, plan->head_dim, plan->num_pages, plan->num_kv_heads,
                              args.cache.stride_page, args.cache.stride_token, args.cache.stride_head) ||
-        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, plan->head_dim, plan->num_pages, plan->num_heads,
+        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, plan->head_dim, plan->num_pages, plan->num_kv_heads,
                              args.cache.stride_page, args.cache.stride_token, args.cache.stride_head))
         return cudaErrorInvalidValue;
     if (plan->head_dim == 128)

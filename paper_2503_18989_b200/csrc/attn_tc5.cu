@@ -177,7 +177,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 
 // What every role needs to know about a unit; all of them decode it the same way.
 struct Unit {
-    int h, r, P, C, row_base, row0, kv_begin, kv_end, part;
+    int h, hk, r, P, C, row_base, row0, kv_begin, kv_end, part;   // h: query head, hk = h / G: the K/V head it reads
     int nq;       // query tiles in use (1 or 2)
     int n_all;    // key tiles of the range
     int n_q0;     // key tiles query tile 0 can see (tile 0 does not see the keys past its own last row)
@@ -187,6 +187,7 @@ __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* _
     const WorkItem it = items[unit / H];
     Unit u;
     u.h = unit % H;
+    u.hk = u.h / a.plan.group;
     u.r = it.req;
     u.P = a.plan.prefix_len[u.r];
     u.C = a.plan.chunk_len[u.r];
@@ -289,7 +290,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                 __syncwarp();
                 if (lane < 16 && pg < npages)
                     tma_load_4d(smem_u32(k_ring) + sk * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0,
-                                u.h, page, &bars->k_full[sk]);
+                                u.hk, page, &bars->k_full[sk]);
                 if (kt >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((kt / kStagesV) & 1) ^ 1, bars, status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -298,7 +299,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                 __syncwarp();
                 if (lane < 16 && pg < npages)
                     tma_load_4d(smem_u32(v_ring) + sv * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0,
-                                u.h, page, &bars->v_full[sv]);
+                                u.hk, page, &bars->v_full[sv]);
             }
         }
         if (!ok) {
@@ -597,9 +598,9 @@ cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStre
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     CUtensorMap mq, mk, mv;
     if (!encode_q_map(&mq, bf16, args.q, plan->total_rows, plan->num_heads) ||
-        !tma_encode_pool_map(&mk, bf16, args.cache.k_pool, kD, plan->num_pages, plan->num_heads, args.cache.stride_page,
+        !tma_encode_pool_map(&mk, bf16, args.cache.k_pool, kD, plan->num_pages, plan->num_kv_heads, args.cache.stride_page,
                              args.cache.stride_token, args.cache.stride_head) ||
-        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, kD, plan->num_pages, plan->num_heads, args.cache.stride_page,
+        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, kD, plan->num_pages, plan->num_kv_heads, args.cache.stride_page,
                              args.cache.stride_token, args.cache.stride_head))
         return cudaErrorInvalidValue;
     // one CTA per SM draws (item, head) units from a counter that is cleared on the stream first

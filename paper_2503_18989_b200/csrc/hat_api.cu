@@ -85,15 +85,20 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     info.prefill_tile_rows = tile_rows;
     info.prefill_kernel = use_tc5 ? 1 : 0;
 
-    // ---- streaming (verify-class) requests: fixed-length key ranges, shortened until the SMs are covered
+    // ---- streaming (verify-class) requests: fixed-length key ranges, shortened until the SMs are covered.
+    // A CTA of the streaming kernel serves one K/V head and 16 (row, query head of the group) pairs.
+    const int group = H / p->num_kv_heads;
+    int max_verify_rows = 0;
     for (int r = 0; r < R; ++r) {
         int C = p->chunk_len[r];
         if (C >= 1 && C <= verify_max_rows) {
             info.num_verify_requests++;
+            max_verify_rows = std::max(max_verify_rows, C);
         } else if (C > verify_max_rows) {
             info.num_prefill_requests++;
         }
     }
+    p->verify_subtiles = std::max(1, ceil_div(max_verify_rows * group, 16));
     int vsplit = env_int("HAT_VERIFY_SPLIT_LEN", 0);
     if (vsplit <= 0) {
         // Long ranges stream best (a CTA's pipeline ramp and its cross-warp merge are paid once per range, and an
@@ -107,7 +112,7 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
                 const int C = p->chunk_len[r];
                 if (C >= 1 && C <= verify_max_rows) n += ceil_div(p->prefix_len[r] + C, len);
             }
-            return n * H;
+            return n * p->num_kv_heads * p->verify_subtiles;
         };
         while (vsplit > 256 && ctas_at(vsplit) < want_ctas) vsplit /= 2;
     }
@@ -190,6 +195,7 @@ static int upload(hat_plan* p) {
     size_t o_vi = blob_append(blob, p->verify_items);
     size_t o_pi = blob_append(blob, p->prefill_items);
     size_t o_mr = blob_append(blob, p->merge_rows);
+    size_t o_tm = blob_append(blob, p->tree_mask);
     std::vector<int32_t> status(4, 0);
     size_t o_st = blob_append(blob, status);
 
@@ -211,7 +217,10 @@ static int upload(hat_plan* p) {
     d.merge_rows = reinterpret_cast<const MergeRow*>(base + o_mr);
     d.status = reinterpret_cast<int32_t*>(base + o_st);
     d.max_pages = p->max_pages;
+    d.tree_mask = p->tree_mask.empty() ? nullptr : reinterpret_cast<const uint32_t*>(base + o_tm);
     d.num_heads = p->num_heads;
+    d.num_kv_heads = p->num_kv_heads;
+    d.group = p->num_heads / p->num_kv_heads;
     d.total_rows = p->total_rows;
     return HAT_OK;
 }
@@ -222,7 +231,7 @@ static int check_call(const hat_cache_desc* cache, const hat_plan* plan) {
     int st = check_cache_geometry(cache);
     if (st != HAT_OK) return st;
     if (cache->dtype != plan->dtype || cache->num_pages != plan->num_pages ||
-        cache->num_kv_heads != plan->num_heads || cache->head_dim != plan->head_dim)
+        cache->num_kv_heads != plan->num_kv_heads || cache->head_dim != plan->head_dim)
         return HAT_ERR_INVALID_ARG;
     if (!cache->k_pool || !cache->v_pool) return HAT_ERR_INVALID_ARG;
     if (!aligned(cache->k_pool, 16) || !aligned(cache->v_pool, 16)) return HAT_ERR_INVALID_ARG;
@@ -265,7 +274,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     if (st != HAT_OK) return st;
     const int R = batch->num_requests;
     if (R < 0 || batch->max_pages < 0 || batch->num_q_heads <= 0) return HAT_ERR_INVALID_ARG;
-    if (batch->num_q_heads != cache->num_kv_heads) return HAT_ERR_UNSUPPORTED;
+    if (batch->num_q_heads % cache->num_kv_heads != 0) return HAT_ERR_UNSUPPORTED;
     if (!batch->cu_chunk) return HAT_ERR_INVALID_ARG;
     if (R > 0 && (!batch->prefix_len || !batch->chunk_len)) return HAT_ERR_INVALID_ARG;
     if (batch->cu_chunk[0] != 0) return HAT_ERR_INVALID_ARG;
@@ -302,7 +311,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     if (!p) return HAT_ERR_INVALID_ARG;
     p->dtype = cache->dtype;
     p->num_pages = cache->num_pages;
-    p->num_heads = cache->num_kv_heads;
+    p->num_heads = batch->num_q_heads;
+    p->num_kv_heads = cache->num_kv_heads;
     p->head_dim = cache->head_dim;
     p->max_pages = batch->max_pages;
     p->num_requests = R;
@@ -323,6 +333,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->chunk_len.assign(batch->chunk_len, batch->chunk_len + R);
     if (batch->block_table && batch->max_pages > 0)
         p->block_table.assign(batch->block_table, batch->block_table + (int64_t)R * batch->max_pages);
+    if (batch->tree_mask) p->tree_mask.assign(batch->tree_mask, batch->tree_mask + total);
     p->row_req.resize(total);
     for (int r = 0; r < R; ++r)
         for (int t = p->cu_chunk[r]; t < p->cu_chunk[r + 1]; ++t) p->row_req[t] = r;
@@ -334,7 +345,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         const int64_t C = p->chunk_len[r], P = p->prefix_len[r];
         if (C == 0) continue;
         p->info.attn_flops += 4 * d * H * (C * P + C * (C + 1) / 2);
-        p->info.kv_read_bytes += 2 * (P + C) * H * d * 2;
+        p->info.kv_read_bytes += 2 * (P + C) * p->num_kv_heads * d * 2;
     }
 
     int num_sms = 148;
@@ -349,7 +360,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     if (const char* k = std::getenv("HAT_PREFILL_KERNEL"))
         if (std::strcmp(k, "mma") == 0) use_tc5 = false;
     if (use_tc5 && !p->host_only)
-        use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
+        use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_kv_heads, cache->stride_page,
                                        cache->stride_token, cache->stride_head);
     p->num_sms = num_sms;
     schedule(p, num_sms, use_tc5);
@@ -358,7 +369,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     if (const char* k = std::getenv("HAT_STREAM_KERNEL"))
         if (std::strcmp(k, "mma") == 0) stream_tma = false;
     if (stream_tma && !p->host_only)
-        stream_tma = stream_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_heads, cache->stride_page,
+        stream_tma = stream_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_kv_heads, cache->stride_page,
                                              cache->stride_token, cache->stride_head);
     p->info.stream_kernel = stream_tma ? 1 : 0;
     // launch-geometry limits: work items index gridDim.y (65535), partial rows and units are 32-bit
@@ -554,11 +565,12 @@ int hat_plan_read_timing(hat_plan* plan, float* ms, int capacity_calls, int* num
 
 int hat_plan_staging_bytes(const hat_plan* plan, size_t* out) {
     if (!plan || !out) return HAT_ERR_INVALID_ARG;
-    const size_t T = plan->total_rows, H = plan->num_heads, d = plan->head_dim;
-    const size_t act16 = (T * H * d * 2 + 255) / 256 * 256;
+    const size_t T = plan->total_rows, H = plan->num_heads, Hkv = plan->num_kv_heads, d = plan->head_dim;
+    const size_t q16 = (T * H * d * 2 + 255) / 256 * 256;
+    const size_t kv16 = (T * Hkv * d * 2 + 255) / 256 * 256;
     const size_t out32 = (T * H * d * 4 + 255) / 256 * 256;
     const size_t lse32 = (T * H * 4 + 255) / 256 * 256;
-    *out = 3 * act16 + out32 + lse32;
+    *out = q16 + 2 * kv16 + out32 + lse32;
     return HAT_OK;
 }
 
@@ -574,20 +586,20 @@ int hat_chunk_attention_host(const hat_cache_desc* cache, const hat_plan* plan, 
     hat_plan_staging_bytes(plan, &need);
     if (!staging || !aligned(staging, 256)) return HAT_ERR_INVALID_ARG;
     if (staging_bytes < need) return HAT_ERR_WORKSPACE_TOO_SMALL;
-    const size_t T = plan->total_rows, H = plan->num_heads, d = plan->head_dim;
-    const size_t act_bytes = T * H * d * 2, out_bytes = T * H * d * 4, lse_bytes = T * H * 4;
-    const size_t act16 = (act_bytes + 255) / 256 * 256, out32 = (out_bytes + 255) / 256 * 256;
+    const size_t T = plan->total_rows, H = plan->num_heads, Hkv = plan->num_kv_heads, d = plan->head_dim;
+    const size_t act_bytes = T * H * d * 2, kv_bytes = T * Hkv * d * 2, out_bytes = T * H * d * 4, lse_bytes = T * H * 4;
+    const size_t q16 = (act_bytes + 255) / 256 * 256, kv16 = (kv_bytes + 255) / 256 * 256, out32 = (out_bytes + 255) / 256 * 256;
     char* base = static_cast<char*>(staging);
     void* dq = base;
-    void* dk = base + act16;
-    void* dv = base + 2 * act16;
-    float* dout = reinterpret_cast<float*>(base + 3 * act16);
-    float* dlse = reinterpret_cast<float*>(base + 3 * act16 + out32);
+    void* dk = base + q16;
+    void* dv = base + q16 + kv16;
+    float* dout = reinterpret_cast<float*>(base + q16 + 2 * kv16);
+    float* dlse = reinterpret_cast<float*>(base + q16 + 2 * kv16 + out32);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     if ((e = cudaMemcpyAsync(dq, q_host, act_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(dk, k_new_host, act_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(dv, v_new_host, act_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
     st = hat_chunk_attention(cache, plan, dq, dk, dv, dout, dlse, sm_scale, workspace, workspace_bytes, stream);
     if (st != HAT_OK) return st;
     if ((e = cudaMemcpyAsync(out_host, dout, out_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);

@@ -41,9 +41,12 @@ struct DevicePlan {
     const WorkItem* verify_items;
     const WorkItem* prefill_items;
     const MergeRow* merge_rows;
+    const uint32_t* tree_mask;      // [T] or null: visible chunk positions of each row of a streaming-class request
     int32_t*        status;         // device status word (0 = ok)
     int32_t         max_pages;
-    int32_t         num_heads;
+    int32_t         num_heads;      // query heads (q, out, lse, partial results)
+    int32_t         num_kv_heads;   // K/V heads (pools, k_new, v_new)
+    int32_t         group;          // query heads per K/V head
     int32_t         total_rows;
 };
 
@@ -80,7 +83,9 @@ struct Timing {
 
 struct hat_plan {
     // geometry the plan was made for
-    int32_t dtype, num_pages, num_heads, head_dim, max_pages, num_requests, total_rows;
+    int32_t dtype, num_pages, num_heads, num_kv_heads, head_dim, max_pages, num_requests, total_rows;   // num_heads: query heads
+    int32_t verify_subtiles;    // 16-row slabs of (row, query head of a group) pairs per streaming work item and K/V head
+    std::vector<uint32_t> tree_mask;
     bool host_only;
     int device;
     int num_sms;

@@ -12,7 +12,7 @@ kv_append_kernel(DevicePlan plan, int64_t stride_page, int64_t stride_token, int
                  int vec_per_head, int64_t total_vecs) {
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total_vecs) return;
-    const int vec_per_row = vec_per_head * plan.num_heads;
+    const int vec_per_row = vec_per_head * plan.num_kv_heads;
     const int t = (int)(idx / vec_per_row);
     const int within = (int)(idx - (int64_t)t * vec_per_row);
     const int h = within / vec_per_head;
@@ -34,7 +34,7 @@ kv_append_kernel(DevicePlan plan, int64_t stride_page, int64_t stride_token, int
 cudaError_t launch_kv_append(const hat_plan* plan, const CacheView& cache, void* k_pool, void* v_pool,
                              const void* k_new, const void* v_new, cudaStream_t stream) {
     const int vec_per_head = plan->head_dim / 8;
-    const int64_t total = (int64_t)plan->total_rows * plan->num_heads * vec_per_head;
+    const int64_t total = (int64_t)plan->total_rows * plan->num_kv_heads * vec_per_head;
     if (total == 0) return cudaSuccess;
     const int threads = 256;
     const int64_t blocks = (total + threads - 1) / threads;

@@ -41,10 +41,11 @@ class DeviceStep:
         spec = cache.spec
         self.cache = cache
         self.step = step
-        self.plan = B.hat_plan_create(cache.desc, spec.num_heads, step.cu_chunk, step.prefix_len, step.chunk_len,
-                                      step.block_table)
+        H = int(step.q.shape[1])                  # query heads; spec.num_heads K/V heads
+        self.plan = B.hat_plan_create(cache.desc, H, step.cu_chunk, step.prefix_len, step.chunk_len,
+                                      step.block_table, tree_mask=getattr(step, "tree_mask", None))
         self.info = B.hat_plan_get_info(self.plan).as_dict()
-        T, H, d = step.total_rows, spec.num_heads, spec.head_dim
+        T, d = step.total_rows, spec.head_dim
         self.q = _dev_u16(step.q, dev)
         self.k_new = _dev_u16(step.k_new, dev)
         self.v_new = _dev_u16(step.v_new, dev)

@@ -80,7 +80,9 @@ def test_plan_rejects_bad_arguments(hat_lib):
     assert _status(_plan, _cache(head_dim=96), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
     assert _status(_plan, _cache(dtype=2), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
     assert _status(_plan, _cache(stride_token=132), [0], [4], [[0]]) == B.HAT_ERR_UNSUPPORTED
-    assert _status(_plan, c, [0], [4], [[0]], H=8) == B.HAT_ERR_UNSUPPORTED       # q heads != kv heads
+    assert _status(_plan, c, [0], [4], [[0]], H=8) == B.HAT_OK                    # two query heads per K/V head
+    assert _status(_plan, c, [0], [4], [[0]], H=6) == B.HAT_ERR_UNSUPPORTED       # not a multiple of the K/V heads
+    assert _status(_plan, c, [0], [4], [[0]], H=2) == B.HAT_ERR_UNSUPPORTED
     # null descriptors
     out = C.c_void_p()
     assert hat_lib.hat_plan_create(None, None, C.byref(out)) == B.HAT_ERR_INVALID_ARG
@@ -153,6 +155,15 @@ def test_schedule_of_prefill_and_mixed_batches(hat_lib):
     assert info["num_prefill_requests"] == 8 and info["num_verify_requests"] == 32
     assert info["total_rows"] == 8 * 512 + 32 * 4
     assert info["max_splits"] <= 32
+
+
+def test_grouped_query_heads_change_the_work_but_not_the_cache_traffic(hat_lib):
+    c = _cache(num_pages=64, H=4, d=128)
+    table = [list(range(40))]
+    one = B.hat_plan_get_info(_plan(c, [600], [4], table, H=4)).as_dict()
+    four = B.hat_plan_get_info(_plan(c, [600], [4], table, H=16)).as_dict()
+    assert four["attn_flops"] == 4 * one["attn_flops"] and four["kv_read_bytes"] == one["kv_read_bytes"]
+    assert four["num_verify_requests"] == 1 and four["total_rows"] == 4
 
 
 def test_long_request_never_exceeds_32_key_ranges(hat_lib):

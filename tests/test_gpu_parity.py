@@ -119,12 +119,14 @@ def test_dtype_headdim_layout_variants(cuda_device, dtype, d, layout):
     _check_full(sc, cuda_device)
 
 
-def _manual(dtype, H, d, prefix, chunk, seed, num_pages=None, table=None, layout="paged"):
-    """Batch with hand-picked prefix/chunk lengths."""
+def _manual(dtype, H, d, prefix, chunk, seed, num_pages=None, table=None, layout="paged", q_group=1, tree=False):
+    """Batch with hand-picked prefix/chunk lengths (H K/V heads, H * q_group query heads)."""
     rng = np.random.Generator(np.random.PCG64(seed))
     if table is None:
         table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=5)
-    st = W._make_step(seed + 100, dtype, H, d, prefix, chunk, table)
+    st = W._make_step(seed + 100, dtype, H, d, prefix, chunk, table, q_heads=H * q_group)
+    if tree:
+        st.tree_mask = W.random_tree_masks(seed + 200, chunk)
     return W._scenario("manual", dtype, H, d, layout, num_pages, [st], seed + 100)
 
 
@@ -369,3 +371,55 @@ def test_verify_rows_are_final_before_the_prompt_chunks_run(cuda_device):
     rows = st.cu_chunk[samples[:, 0]] + samples[:, 1]
     assert_parity(go[rows, samples[:, 2]], wo, "verify rows out")
     assert_parity(gl[rows, samples[:, 2]], wl, "verify rows lse")
+
+
+# ----------------------------------------------------------------------------
+# grouped query heads and token trees
+# ----------------------------------------------------------------------------
+_GQA_PREFIX = [40, 0, 33, 250, 5, 1000, 77, 0, 1023, 600, 17]
+_GQA_CHUNK = [0, 1, 8, 16, 17, 3, 65, 129, 7, 300, 12]
+
+
+@pytest.mark.parametrize("dtype,d,group,layout", [("fp16", 128, 2, "paged"), ("bf16", 128, 4, "paged"),
+                                                  ("fp16", 64, 8, "paged"), ("bf16", 64, 3, "contiguous"),
+                                                  ("fp16", 128, 5, "contiguous")])
+def test_grouped_query_heads(cuda_device, dtype, d, group, layout):
+    """G query heads share each K/V head: every chunk class, chunk rows x G both below and above one 16-row
+    slab, q / out / lse with G times the heads of the pools."""
+    sc = _manual(dtype, 2, d, _GQA_PREFIX, _GQA_CHUNK, 31 + group, layout=layout, q_group=group)
+    got, want = _check_full(sc, cuda_device)
+    assert got[0][0].shape == (sum(_GQA_CHUNK), 2 * group, d)
+
+
+@pytest.mark.parametrize("dtype,d,group", [("fp16", 128, 1), ("bf16", 128, 4), ("bf16", 64, 2)])
+def test_token_trees(cuda_device, dtype, d, group):
+    """Random token trees on every short chunk (1..16 rows, empty and mid-page prefixes, ranges cut by the
+    scheduler), causal long chunks in the same batch."""
+    sc = _manual(dtype, 2, d, _GQA_PREFIX + [9000], _GQA_CHUNK + [16], 41 + group, q_group=group, tree=True)
+    st = sc.steps[0]
+    assert any(int(w) != (2 << i) - 1 for r in range(st.num_requests) if st.chunk_len[r] <= 16
+               for i, w in enumerate(st.tree_mask[st.cu_chunk[r]:st.cu_chunk[r + 1]])), "the trees must not all be chains"
+    _check_full(sc, cuda_device)
+
+
+def test_tree_row_that_sees_nothing_and_rows_that_see_later_positions(cuda_device):
+    from paper_2503_18989_b200 import runner
+    sc = _manual("fp16", 2, 128, [0, 20], [3, 4], 51, q_group=2)
+    st = sc.steps[0]
+    st.tree_mask = np.asarray([0b000, 0b110, 0b101, 0b1000, 0b0011, 0b1111, 0b0100], np.uint32)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    ds.attend()
+    go, gl = ds.results()
+    kp, vp, want = oracle_replay(sc)
+    wo, wl = want[0]
+    assert np.all(go[0] == 0) and np.all(gl[0] == -np.inf) and np.all(wl[0] == -np.inf)
+    assert_parity(go[1:], wo[1:], "tree out")
+    assert_parity(gl[1:], wl[1:], "tree lse")
+
+
+@pytest.mark.parametrize("which", ["stream", "tile"])
+def test_grouped_heads_and_trees_on_the_mma_sync_kernels(cuda_device, which, monkeypatch):
+    monkeypatch.setenv("HAT_STREAM_KERNEL" if which == "stream" else "HAT_PREFILL_KERNEL", "mma")
+    sc = _manual("bf16", 2, 128, _GQA_PREFIX, _GQA_CHUNK, 61, q_group=4, tree=True)
+    _check_full(sc, cuda_device)
