@@ -48,12 +48,13 @@ def load_peaks():
 # every visible K and V row read once per head)
 # ----------------------------------------------------------------------------
 def step_work(cache, st):
-    H, d, e = cache.num_heads, cache.head_dim, 2
+    Hkv, d, e = cache.num_heads, cache.head_dim, 2
+    H = int(st.q.shape[1])                      # query heads (= K/V heads in the paper's models)
     P = st.prefix_len.astype(np.int64)
     Cn = st.chunk_len.astype(np.int64)
-    pairs = Cn * P + Cn * (Cn + 1) // 2
+    pairs = Cn * P + Cn * (Cn + 1) // 2         # causal count, also when a token tree thins the chunk's own keys
     flops = 4 * d * H * pairs
-    kv_bytes = 2 * (P + Cn) * H * d * e * (Cn > 0)
+    kv_bytes = 2 * (P + Cn) * Hkv * d * e * (Cn > 0)
     io_bytes = Cn * H * d * e + Cn * H * d * 4 + Cn * H * 4            # q in, out + lse out
     short = (Cn > 0) & (Cn <= VERIFY_MAX_ROWS)
     long_ = Cn > VERIFY_MAX_ROWS
@@ -62,7 +63,7 @@ def step_work(cache, st):
         "flops": int(flops.sum()),
         "tile_flops": int(flops[long_].sum()), "tile_bytes": int((kv_bytes + io_bytes)[long_].sum()),
         "stream_flops": int(flops[short].sum()), "stream_bytes": int((kv_bytes + io_bytes)[short].sum()),
-        "append_bytes": int(4 * T * H * d * e),
+        "append_bytes": int(4 * T * Hkv * d * e),
         "kv_bytes": int(kv_bytes.sum()),
         "rows": T,
     }
@@ -162,7 +163,7 @@ def lookup_traffic(kernel: str, workload: str):
 
 def pick_oracle_sample(cache, st, rng, target_flops):
     """(request, row, head) units drawn uniformly over all (row, head) pairs until ~target_flops."""
-    H, d = cache.num_heads, cache.head_dim
+    H, d = int(st.q.shape[1]), cache.head_dim
     live = np.nonzero(st.chunk_len > 0)[0]
     rows_req = np.repeat(live, st.chunk_len[live])
     rows_i = np.concatenate([np.arange(int(st.chunk_len[r])) for r in live])
@@ -193,12 +194,22 @@ def time_oracle(sc, budget_s, seed=0):
         units, fl
 
 
+def make_workload(args, seed=None):
+    """The named workload; --q-group / --tree reach the two workloads that have decode-phase requests."""
+    kw = {} if seed is None else {"seed": seed}
+    if args.q_group != 1 or args.tree:
+        if args.workload not in ("spec_verify", "mixed_13b"):
+            raise SystemExit("--q-group and --tree apply to spec_verify and mixed_13b only")
+        kw.update(q_group=args.q_group, tree=args.tree)
+    return W.WORKLOADS[args.workload](**kw)
+
+
 def run_reference(args, rank):
     """Reference arm: the CPU oracle, as it stands, on the host cores."""
     if rank != 0:
         return
     from oracle import hat_oracle as O
-    sc = W.WORKLOADS[args.workload]()
+    sc = make_workload(args)
     st = sc.steps[-1]
     for s in sc.steps:
         O.kv_append(sc.cache, sc.k_pool, sc.v_pool, s)
@@ -234,6 +245,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="mixed_13b", choices=sorted(W.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--q-group", type=int, default=1,
+                    help="query heads per K/V head (spec_verify and mixed_13b only; the paper's models have 1)")
+    ap.add_argument("--tree", action="store_true",
+                    help="token trees instead of linear drafts on the short chunks (spec_verify and mixed_13b only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
     args = ap.parse_args()
@@ -278,7 +293,7 @@ def main():
     peaks, peak_kind = load_peaks()
 
     # ---- inputs: one replica of the batch per rank (seeded; different values per rank)
-    sc = W.WORKLOADS[args.workload](seed=replica_seed(args.workload, rank))
+    sc = make_workload(args, seed=replica_seed(args.workload, rank))
     cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, device)
     steps = [runner.DeviceStep(cache, st) for st in sc.steps]
     works = [step_work(sc.cache, st) for st in sc.steps]
@@ -340,7 +355,7 @@ def main():
     Ke = max(1, min(K, 100))
     host = []
     for ds, st in zip(steps, sc.steps):
-        T, H, d = st.total_rows, sc.cache.num_heads, sc.cache.head_dim
+        T, H, d = st.total_rows, int(st.q.shape[1]), sc.cache.head_dim
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
         nb = B.hat_plan_staging_bytes(ds.plan)
         host.append((pin(st.q), pin(st.k_new), pin(st.v_new),
@@ -364,8 +379,8 @@ def main():
     e2e_ms = e0.elapsed_time(e1)
     barrier()
     sampler.stop()
-    h2d = sum(3 * st.q.nbytes for st in sc.steps)
-    d2h = sum(st.total_rows * sc.cache.num_heads * (sc.cache.head_dim + 1) * 4 for st in sc.steps)
+    h2d = sum(st.q.nbytes + st.k_new.nbytes + st.v_new.nbytes for st in sc.steps)
+    d2h = sum(st.total_rows * int(st.q.shape[1]) * (sc.cache.head_dim + 1) * 4 for st in sc.steps)
 
     # ---- max over ranks
     elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e_ms], world, device)
@@ -414,7 +429,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": sc.cache.dtype + " in, f32 accumulate",
             "data": "synthetic",
             "config": {"workload": sc.name, "requests": int(sc.steps[-1].num_requests), "rows": total["rows"],
-                       "heads": sc.cache.num_heads, "head_dim": sc.cache.head_dim, "page_size": 16,
+                       "heads": int(sc.steps[-1].q.shape[1]), "kv_heads": sc.cache.num_heads,
+                       "token_trees": bool(args.tree), "head_dim": sc.cache.head_dim, "page_size": 16,
                        "calls_per_step": len(sc.steps), "kv_resident_bytes": int(kv_resident),
                        "l2": "flushed between steps" if flush_l2 else "KV working set larger than L2",
                        "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
