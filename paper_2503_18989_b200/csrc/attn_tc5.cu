@@ -17,6 +17,8 @@
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512).  P_t(j) overwrites S_t(j) in place (16-bit pairs in
 // columns [0,64), the bf16 rounding remainder in [64,128)); S_t(j+1) is issued after P_t V(j) by the same thread, and
 // tcgen05 executes one thread's MMAs in issue order, so no extra barrier guards the reuse.
+// A unit of at most 128 rows uses both column pairs for the SAME query tile: two chains over alternating key tiles,
+// merged by the first chain's warpgroup when the unit ends (see Unit::split).
 // Every wait is bounded (about a second by default); a wait that gives up sets the plan's status word, raises a
 // CTA-wide abort flag that all other waits observe, and the CTA still frees its TMEM and exits normally.
 #include <cuda.h>
@@ -24,6 +26,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "hat_internal.h"
 #include "tma_desc.h"
@@ -47,13 +50,16 @@ struct __align__(8) Barriers {
     uint64_t v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], p_ready[2], o_done[2], o_free[2];   // per query tile
     uint64_t unit_full[2], unit_empty[2];                   // two-slot queue of work units, producer -> other roles
+    uint64_t x_ready;                                       // split units: chain 1's (reference maximum, row sum) are in xchg
     uint64_t drain;
     long long wait_cycles;                                  // bound of every wait below
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile int unit_slot[2];                              // unit index, or -1 when the work has run out
+    float2 xchg[kRows];                                     // split units: per row, chain 1's reference maximum and row sum
 };
-constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + kStagesK + kStagesV) + 256;
+constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + kStagesK + kStagesV) + sizeof(Barriers);
+static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 constexpr int kThreads = 320;   // producer warp, MMA warp, two softmax warpgroups
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -141,6 +147,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
         ::"r"(taddr), HAT_W32(r, 0), HAT_W32(r, 8), HAT_W32(r, 16), HAT_W32(r, 24) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+        : HAT_R32(r, 0), HAT_R32(r, 8)
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
@@ -181,6 +193,14 @@ struct Unit {
     int nq;       // query tiles in use (1 or 2)
     int n_all;    // key tiles of the range
     int n_q0;     // key tiles query tile 0 can see (tile 0 does not see the keys past its own last row)
+    // A unit with a single query tile would leave the second accumulator pair and warpgroup idle and the tensor
+    // pipe waiting through every softmax.  It runs as two chains instead: chain t takes key tiles t, t+2, t+4, ... with
+    // the same Q tile, and the two partial results (disjoint key sets) are merged when the unit ends.
+    bool split;
+    int n_t0, n_t1;   // key tiles of chain (or query tile) 0 and 1
+    __device__ __forceinline__ int n_t(int t) const { return t == 0 ? n_t0 : n_t1; }
+    // key tile of step s of chain t
+    __device__ __forceinline__ int tile_of(int t, int s) const { return split ? 2 * s + t : s; }
 };
 __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* __restrict__ items, int unit) {
     const int H = a.plan.num_heads;
@@ -197,6 +217,9 @@ __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* _
     u.n_all = (u.kv_end - u.kv_begin + kKeys - 1) / kKeys;
     const int end0 = min(u.kv_end, u.P + u.row0 + kRows);
     u.n_q0 = u.nq == 1 ? u.n_all : max(0, (end0 - u.kv_begin + kKeys - 1) / kKeys);
+    u.split = u.nq == 1;
+    u.n_t0 = u.split ? (u.n_all + 1) / 2 : u.n_q0;
+    u.n_t1 = u.split ? u.n_all / 2 : (u.nq == 2 ? u.n_all : 0);
     return u;
 }
 
@@ -229,6 +252,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
             mbar_init(&bars->unit_full[s], 1);
             mbar_init(&bars->unit_empty[s], 1 + 8);              // the MMA thread and every softmax warp
         }
+        mbar_init(&bars->x_ready, 4);
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
         bars->wait_cycles = a.wait_cycles;
@@ -328,76 +352,83 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                 const Unit u = decode_unit(a, items, unit);
                 ok = mbar_wait(&bars->q_full, un & 1, bars, status);
                 if (!ok) break;
-                int k_ready = -1, v_ready = -1;       // last K / V tile of this unit known to have landed
-                // S_t(j) = Q_t K(j)^T into TMEM columns [128 t, 128 t + 128)
-                auto issue_s = [&](int qt, int j) {
-                    const int kt = kt_base + j, st = kt % kStagesK;
-                    if (k_ready < j) {
-                        ok = mbar_wait(&bars->k_full[st], (kt / kStagesK) & 1, bars, status);
-                        k_ready = j;
+                // the two kinds of unit get their own copy of the issue loop: every instruction of this thread counts
+                auto run_unit = [&](auto split_tag) {
+                    constexpr bool SPLIT = decltype(split_tag)::value;
+                    int k_ready = -1, v_ready = -1;       // last K / V tile of this unit known to have landed
+                    // S_t(s) = Q K(j)^T into TMEM columns [128 t, 128 t + 128), j = the key tile of step s of chain / tile t
+                    auto issue_s = [&](int qt, int sidx) {
+                        const int j = SPLIT ? 2 * sidx + qt : sidx;
+                        const int kt = kt_base + j, st = kt % kStagesK;
+                        if (k_ready < j) {
+                            ok = mbar_wait(&bars->k_full[st], (kt / kStagesK) & 1, bars, status);
+                            k_ready = j;
+                            if (!ok) return;
+                        }
+                        const uint32_t q_addr = smem_u32(q_tiles) + (SPLIT ? 0 : qt) * kTileBytes;
+                        const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
+                        tc_fence_after();
+    #pragma unroll
+                        for (int ks = 0; ks < kD / 16; ++ks) {
+                            const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
+                            mma_ss(tmem + qt * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                        }
+                        tc_commit(&bars->s_full[qt]);
+                        if (SPLIT || qt == u.nq - 1) {
+                            tc_commit(&bars->k_empty[st]);                       // the last reader of this K tile
+                            if (j == u.n_all - 1) tc_commit(&bars->q_empty);     // and the unit's last read of the Q tiles
+                        }
+                    };
+                    // O_t (+)= P_t V(j); P sits in the columns S_t was computed in
+                    auto issue_pv = [&](int qt, int sidx) {
+                        const int j = SPLIT ? 2 * sidx + qt : sidx;
+                        const int kt = kt_base + j, st = kt % kStagesV;
+                        if (v_ready < j) {
+                            ok = mbar_wait(&bars->v_full[st], (kt / kStagesV) & 1, bars, status);
+                            v_ready = j;
+                            if (!ok) return;
+                        }
+                        if (sidx == 0 && o_busy[qt]) {
+                            // the accumulator still holds the previous unit: wait until its rows are in registers
+                            ok = mbar_wait(&bars->o_free[qt], f_cnt[qt] & 1, bars, status);
+                            ++f_cnt[qt];
+                            o_busy[qt] = false;
+                            if (!ok) return;
+                        }
+                        ok = mbar_wait(&bars->p_ready[qt], p_cnt[qt] & 1, bars, status);
+                        ++p_cnt[qt];
                         if (!ok) return;
-                    }
-                    const uint32_t q_addr = smem_u32(q_tiles) + qt * kTileBytes;
-                    const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
-                        mma_ss(tmem + qt * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
-                    }
-                    tc_commit(&bars->s_full[qt]);
-                    if (qt == u.nq - 1) {
-                        tc_commit(&bars->k_empty[st]);                       // the last reader of this K tile
-                        if (j == u.n_all - 1) tc_commit(&bars->q_empty);     // and the unit's last read of the Q tiles
+                        tc_fence_after();
+                        const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
+                        const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
+    #pragma unroll
+                        for (int ks = 0; ks < kKeys / 16; ++ks) {
+                            // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
+                            const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
+                            mma_ts(to, tp + ks * 8, vdesc, idesc_o, (sidx > 0) || (ks > 0));
+                            if constexpr (BF16) mma_ts(to, tp + 64 + ks * 8, vdesc, idesc_o, true);
+                        }
+                        tc_commit(&bars->o_done[qt]);
+                        if (SPLIT || qt == u.nq - 1) tc_commit(&bars->v_empty[st]);
+                    };
+                    if (u.n_t0 > 0) issue_s(0, 0);
+                    if (ok && u.n_t1 > 0) issue_s(1, 0);
+                    for (int sidx = 0; sidx < max(u.n_t0, u.n_t1) && ok; ++sidx) {
+                        // tile 0's P V, then at once its next S: the tensor pipe works on them while tile 1's softmax runs
+                        if (sidx < u.n_t0) {
+                            issue_pv(0, sidx);
+                            if (ok && sidx + 1 < u.n_t0) issue_s(0, sidx + 1);
+                        }
+                        if (ok && sidx < u.n_t1) {
+                            issue_pv(1, sidx);
+                            if (ok && sidx + 1 < u.n_t1) issue_s(1, sidx + 1);
+                        }
                     }
                 };
-                // O_t (+)= P_t(j) V(j); P sits in the columns S_t(j) was computed in
-                auto issue_pv = [&](int qt, int j) {
-                    const int kt = kt_base + j, st = kt % kStagesV;
-                    if (v_ready < j) {
-                        ok = mbar_wait(&bars->v_full[st], (kt / kStagesV) & 1, bars, status);
-                        v_ready = j;
-                        if (!ok) return;
-                    }
-                    if (j == 0 && o_busy[qt]) {
-                        // the accumulator still holds the previous unit: wait until its rows are in registers
-                        ok = mbar_wait(&bars->o_free[qt], f_cnt[qt] & 1, bars, status);
-                        ++f_cnt[qt];
-                        o_busy[qt] = false;
-                        if (!ok) return;
-                    }
-                    ok = mbar_wait(&bars->p_ready[qt], p_cnt[qt] & 1, bars, status);
-                    ++p_cnt[qt];
-                    if (!ok) return;
-                    tc_fence_after();
-                    const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
-                    const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
-#pragma unroll
-                    for (int ks = 0; ks < kKeys / 16; ++ks) {
-                        // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
-                        const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
-                        mma_ts(to, tp + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));
-                        if constexpr (BF16) mma_ts(to, tp + 64 + ks * 8, vdesc, idesc_o, true);
-                    }
-                    tc_commit(&bars->o_done[qt]);
-                    if (qt == u.nq - 1) tc_commit(&bars->v_empty[st]);
-                };
-                if (u.n_q0 > 0) issue_s(0, 0);
-                if (ok && u.nq == 2) issue_s(1, 0);
-                for (int j = 0; j < u.n_all && ok; ++j) {
-                    // tile 0's P V(j), then at once its next S: the tensor pipe works on them while tile 1's softmax runs
-                    if (j < u.n_q0) {
-                        issue_pv(0, j);
-                        if (ok && j + 1 < u.n_q0) issue_s(0, j + 1);
-                    }
-                    if (ok && u.nq == 2) {
-                        issue_pv(1, j);
-                        if (ok && j + 1 < u.n_all) issue_s(1, j + 1);
-                    }
-                }
+                if (u.split) run_unit(std::true_type{}); else run_unit(std::false_type{});
                 // a unit in which a tile had no keys leaves that tile's earlier hand-over pending
-                if (u.n_q0 > 0) o_busy[0] = true;
-                if (u.nq == 2) o_busy[1] = true;
+                if (u.n_t0 > 0) o_busy[0] = true;
+                if (u.n_t1 > 0) o_busy[1] = true;
                 kt_base += u.n_all;
             }
             if (!ok) {
@@ -418,7 +449,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
         const int wg_tid = (int)threadIdx.x - 64 - qt * 128;
         const float sc = a.scale_log2;
         int kt_base = 0;                                    // K/V tiles of the units before this one
-        int s_cnt = 0, o_cnt = 0;                           // completions of s_full[qt] / o_done[qt] consumed so far
+        int s_cnt = 0, o_cnt = 0, x_cnt = 0;                // completions of s_full[qt] / o_done[qt] / x_ready consumed so far
         bool ok = true;
         for (int un = 0; ok; ++un) {
             const int slot = un & 1;
@@ -429,12 +460,13 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
             if (lane == 0) mbar_arrive(&bars->unit_empty[slot]);
             if (unit < 0) break;
             const Unit u = decode_unit(a, items, unit);
-            if (qt < u.nq) {
-                const int n_mine = (qt == 0) ? u.n_q0 : u.n_all;
-                const int i_row = u.row0 + qt * kRows + t;   // row inside the chunk
+            if (qt < u.nq || u.split) {
+                const int n_mine = u.n_t(qt);
+                const int i_row = u.row0 + (u.split ? 0 : qt * kRows) + t;   // row inside the chunk
                 const int last_key = min(u.P + i_row, u.kv_end - 1);
                 float m_used = -INFINITY, l = 0.f;           // in units of scale_log2
-                for (int j = 0; j < n_mine; ++j) {
+                for (int sidx = 0; sidx < n_mine; ++sidx) {
+                    const int j = u.tile_of(qt, sidx);       // key tile of this step
                     const int kb = u.kv_begin + j * kKeys;
                     ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[qt], s_cnt & 1, bars, status));
                     ++s_cnt;
@@ -491,7 +523,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
 
                     // O may only be rescaled once the previous P V product has finished; waiting here every tile (it
                     // has long completed by now) also keeps this thread's count of the barrier's phases exact
-                    if (j > 0) {
+                    if (sidx > 0) {
                         ok = __all_sync(0xffffffffu, mbar_wait(&bars->o_done[qt], o_cnt & 1, bars, status));
                         ++o_cnt;
                         if (!ok) break;
@@ -536,26 +568,65 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                     ++o_cnt;
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) tmem_ld32(tm_o + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
-                    tmem_ld_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->o_free[qt]);
-                } else {
-#pragma unroll
-                    for (int k = 0; k < kD; ++k) o[k] = 0.f;
                 }
-                if (i_row < u.C) {
-                    const float inv = l > 0.f ? 1.f / l : 0.f;
-                    float* obase; float* lbase; int64_t orow;
-                    if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
-                    else { obase = a.part_out; lbase = a.part_lse; orow = u.part + qt * kRows + t; }
-                    float* dst = obase + (orow * H + u.h) * kD;
+                if (u.split && qt == 1) {
+                    // second chain of a split unit: its accumulator is complete; publish the row's reference maximum
+                    // and sum, the first chain's warpgroup reads the accumulator itself (same TMEM lanes) and stores
+                    if (n_mine > 0) {
+                        bars->xchg[t] = make_float2(m_used, l);
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->x_ready);
+                    }
+                } else {
+                    if (n_mine > 0) {
 #pragma unroll
-                    for (int k = 0; k < kD; k += 4)
-                        *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
-                    lbase[orow * H + u.h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                        for (int c = 0; c < 4; ++c) tmem_ld32(tm_o + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
+                        tmem_ld_wait();
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < kD; ++k) o[k] = 0.f;
+                    }
+                    if (u.split && u.n_t1 > 0) {
+                        // merge the second chain (disjoint keys): weights 2^(m_t - m), sums and accumulators add up
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_ready, x_cnt & 1, bars, status));
+                        ++x_cnt;
+                        if (!ok) break;
+                        tc_fence_after();
+                        const float2 other = bars->xchg[t];
+                        const float m_new = fmaxf(m_used, other.x);
+                        const float w0 = (m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_new);
+                        const float w1 = (other.x == -INFINITY) ? 0.f : fast_exp2(other.x - m_new);
+                        l = l * w0 + other.y * w1;
+                        m_used = m_new;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t o1[16];
+                            tmem_ld16(tm_o + 128 + c * 16, o1);      // the second chain's accumulator: next 128 columns
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) o[c * 16 + k] = o[c * 16 + k] * w0 + __uint_as_float(o1[k]) * w1;
+                        }
+                    }
+                    if (n_mine > 0 || (u.split && u.n_t1 > 0)) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (n_mine > 0) mbar_arrive(&bars->o_free[qt]);
+                            if (u.split && u.n_t1 > 0) mbar_arrive(&bars->o_free[1]);
+                        }
+                    }
+                    if (i_row < u.C) {
+                        const float inv = l > 0.f ? 1.f / l : 0.f;
+                        float* obase; float* lbase; int64_t orow;
+                        if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
+                        else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
+                        float* dst = obase + (orow * H + u.h) * kD;
+#pragma unroll
+                        for (int k = 0; k < kD; k += 4)
+                            *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
+                        lbase[orow * H + u.h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                    }
                 }
             }
             kt_base += u.n_all;
