@@ -337,6 +337,10 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
             constexpr uint32_t fmt = BF16 ? 1u : 0u;
             constexpr uint32_t idesc_s = make_idesc(fmt, 0, kRows, kKeys);   // Q (K-major) x K (K-major)
             constexpr uint32_t idesc_o = make_idesc(fmt, 1, kRows, kD);      // P (TMEM)    x V (MN-major)
+            // matrix descriptors of Q tile 0 and of slot 0 of each ring, built once
+            const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles), 16, 1024);
+            const uint64_t k_desc0 = smem_desc(smem_u32(k_ring), 16, 1024);
+            const uint64_t v_desc0 = smem_desc(smem_u32(v_ring), kSlabBytes, 1024);
             bool ok = true;
             int kt_base = 0;                          // K/V tiles of the units before this one
             int p_cnt[2] = {0, 0};                    // completions of p_ready[t] consumed so far
@@ -365,13 +369,14 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                             k_ready = j;
                             if (!ok) return;
                         }
-                        const uint32_t q_addr = smem_u32(q_tiles) + (SPLIT ? 0 : qt) * kTileBytes;
-                        const uint32_t k_addr = smem_u32(k_ring) + st * kTileBytes;
+                        // descriptors of the first 16 columns; the others differ in the address field only
+                        const uint64_t qd = q_desc0 + (uint64_t)((SPLIT ? 0 : qt) * (kTileBytes >> 4));
+                        const uint64_t kd = k_desc0 + (uint64_t)(st * (kTileBytes >> 4));
                         tc_fence_after();
-    #pragma unroll
+#pragma unroll
                         for (int ks = 0; ks < kD / 16; ++ks) {
-                            const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;   // 16 columns = 32 bytes inside a slab row
-                            mma_ss(tmem + qt * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+                            const uint32_t off = ((ks >> 2) * kSlabBytes + (ks & 3) * 32) >> 4;   // 16 columns = 32 bytes inside a slab row
+                            mma_ss(tmem + qt * 128, qd + off, kd + off, idesc_s, ks > 0);
                         }
                         tc_commit(&bars->s_full[qt]);
                         if (SPLIT || qt == u.nq - 1) {
@@ -399,12 +404,12 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         ++p_cnt[qt];
                         if (!ok) return;
                         tc_fence_after();
-                        const uint32_t v_addr = smem_u32(v_ring) + st * kTileBytes;
+                        const uint64_t vd = v_desc0 + (uint64_t)(st * (kTileBytes >> 4));
                         const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
-    #pragma unroll
+#pragma unroll
                         for (int ks = 0; ks < kKeys / 16; ++ks) {
                             // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
-                            const uint64_t vdesc = smem_desc(v_addr + ks * 2048, kSlabBytes, 1024);
+                            const uint64_t vdesc = vd + (uint64_t)((ks * 2048) >> 4);
                             mma_ts(to, tp + ks * 8, vdesc, idesc_o, (sidx > 0) || (ks > 0));
                             if constexpr (BF16) mma_ts(to, tp + 64 + ks * 8, vdesc, idesc_o, true);
                         }
