@@ -158,6 +158,10 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
         ::"r"(taddr), HAT_W32(r, 0), HAT_W32(r, 8) : "memory");
 }
+__device__ __forceinline__ void st_global_v8(float* p, float a, float b, float c, float d, float e, float f, float g, float h) {
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
+                 ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d), "f"(e), "f"(f), "f"(g), "f"(h) : "memory");
+}
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
@@ -453,6 +457,8 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
         const uint32_t tm_s = tmem + qt * 128 + lane_sel, tm_o = tmem + 256 + qt * 128 + lane_sel;
         const int wg_tid = (int)threadIdx.x - 64 - qt * 128;
         const float sc = a.scale_log2;
+        // rows are 512 bytes apart at least, so a 32-byte aligned base keeps every 32-byte store aligned
+        const bool wide_stores = ((reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.part_out)) & 31) == 0;
         int kt_base = 0;                                    // K/V tiles of the units before this one
         int s_cnt = 0, o_cnt = 0, x_cnt = 0;                // completions of s_full[qt] / o_done[qt] / x_ready consumed so far
         bool ok = true;
@@ -627,9 +633,18 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
                         else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
                         float* dst = obase + (orow * H + u.h) * kD;
+                        // a thread stores its whole row; 32-byte stores fill a sector each (half as many sector writes as
+                        // 16-byte ones, and the sector rate is what bounds this part)
+                        if (wide_stores) {
 #pragma unroll
-                        for (int k = 0; k < kD; k += 4)
-                            *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
+                            for (int k = 0; k < kD; k += 8)
+                                st_global_v8(dst + k, o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv, o[k + 4] * inv,
+                                             o[k + 5] * inv, o[k + 6] * inv, o[k + 7] * inv);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < kD; k += 4)
+                                *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
+                        }
                         lbase[orow * H + u.h] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
                     }
                 }
