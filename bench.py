@@ -247,6 +247,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--q-group", type=int, default=1,
                     help="query heads per K/V head (spec_verify and mixed_13b only; the paper's models have 1)")
+    ap.add_argument("--out16", action="store_true",
+                    help="device-resident timing through hat_chunk_attention_out16 (output in the cache's 16-bit type); "
+                         "the e2e leg keeps the fp32 host entry point")
     ap.add_argument("--tree", action="store_true",
                     help="token trees instead of linear drafts on the short chunks (spec_verify and mixed_13b only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -305,7 +308,10 @@ def main():
 
     def one_step():
         for ds in steps:
-            ds.attend(fused_append=True, stream=stream)
+            if args.out16:
+                ds.attend16(fused_append=True, stream=stream)
+            else:
+                ds.attend(fused_append=True, stream=stream)
 
     for _ in range(args.warmup):
         one_step()
@@ -430,7 +436,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": sc.name, "requests": int(sc.steps[-1].num_requests), "rows": total["rows"],
                        "heads": int(sc.steps[-1].q.shape[1]), "kv_heads": sc.cache.num_heads,
-                       "token_trees": bool(args.tree), "head_dim": sc.cache.head_dim, "page_size": 16,
+                       "token_trees": bool(args.tree), "out": "16-bit" if args.out16 else "f32", "head_dim": sc.cache.head_dim, "page_size": 16,
                        "calls_per_step": len(sc.steps), "kv_resident_bytes": int(kv_resident),
                        "l2": "flushed between steps" if flush_l2 else "KV working set larger than L2",
                        "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},

@@ -196,6 +196,20 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same step with `out` in the cache's 16-bit type (what the output
+ * projection of the decoder layer, Sec. 2.1, consumes): the fp32 result is
+ * rounded to nearest once, when a final row is written; partial rows in the
+ * workspace and lse stay fp32.  The paper fixes no output precision; this
+ * entry point is an addition next to the fp32 one.
+ *   out16            device [T][num_q_heads][head_dim], cache dtype, 16-byte aligned
+ * All other arguments and errors as hat_chunk_attention.
+ */
+int hat_chunk_attention_out16(const hat_cache_desc* cache, const hat_plan* plan, const void* q,
+                              const void* k_new, const void* v_new,
+                              void* out16, float* lse, float sm_scale,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The same step for a caller whose activations live in HOST memory (pinned
  * memory makes the copies asynchronous).  Copies q, k_new, v_new to `staging`,
  * appends, attends, copies out and lse back, all on `stream`, and returns

@@ -32,7 +32,8 @@ DTYPE_CODE = {"fp16": HAT_DTYPE_FP16, "bf16": HAT_DTYPE_BF16}
 EXPORTS = [
     "hat_status_string", "hat_version", "hat_last_cuda_error", "hat_launch_count",
     "hat_plan_create", "hat_plan_get_info", "hat_plan_workspace_bytes", "hat_plan_destroy",
-    "hat_kv_append", "hat_chunk_attention", "hat_plan_staging_bytes", "hat_chunk_attention_host",
+    "hat_kv_append", "hat_chunk_attention", "hat_chunk_attention_out16", "hat_plan_staging_bytes",
+    "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
     "hat_verify_attention_static", "hat_plan_set_wait_limit",
     "hat_plan_verify_event", "hat_plan_wait_verify",
@@ -111,6 +112,8 @@ def lib() -> C.CDLL:
         L.hat_kv_append.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, vp]
         L.hat_chunk_attention.restype = i32
         L.hat_chunk_attention.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, vp, vp, vp, C.c_float, vp, sz, vp]
+        L.hat_chunk_attention_out16.restype = i32
+        L.hat_chunk_attention_out16.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, vp, vp, vp, C.c_float, vp, sz, vp]
         L.hat_plan_staging_bytes.restype = i32
         L.hat_plan_staging_bytes.argtypes = [vp, C.POINTER(sz)]
         L.hat_chunk_attention_host.restype = i32
@@ -256,6 +259,13 @@ def hat_chunk_attention(cache: hat_cache_desc, plan, q, k_new, v_new, out, lse, 
     _check(lib().hat_chunk_attention(C.byref(cache), _h(plan), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                                      _ptr(lse), float(sm_scale), _ptr(workspace), int(workspace_bytes),
                                      stream or None), "hat_chunk_attention")
+
+
+def hat_chunk_attention_out16(cache: hat_cache_desc, plan, q, k_new, v_new, out16, lse, sm_scale: float = 0.0,
+                              workspace=None, workspace_bytes: int = 0, stream: int = 0) -> None:
+    _check(lib().hat_chunk_attention_out16(C.byref(cache), _h(plan), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out16),
+                                           _ptr(lse), C.c_float(sm_scale), _ptr(workspace), workspace_bytes,
+                                           stream or None), "hat_chunk_attention_out16")
 
 
 def hat_chunk_attention_host(cache: hat_cache_desc, plan, q_host, k_new_host, v_new_host, out_host, lse_host,

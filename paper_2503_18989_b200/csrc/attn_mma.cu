@@ -376,18 +376,23 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
         obase = a.part_out; lbase = a.part_lse;
         r0 = item.part + (i0 - item.row0); r1 = item.part + (i1 - item.row0);
     }
+    const bool to16 = item.part < 0 && a.out16 != nullptr;      // final rows in the 16-bit output type
     if (i0 < C) {
-        float* dst = obase + (r0 * H + h) * D + 2 * t4;
+        const int64_t at = (r0 * H + h) * D + 2 * t4;
 #pragma unroll
-        for (int n = 0; n < ON; ++n)
-            *reinterpret_cast<float2*>(dst + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+        for (int n = 0; n < ON; ++n) {
+            if (to16) *reinterpret_cast<uint32_t*>(static_cast<uint16_t*>(a.out16) + at + n * 8) = pack_out16(o[n][0] * inv0, o[n][1] * inv0, a.out16_bf16);
+            else *reinterpret_cast<float2*>(obase + at + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+        }
         if (t4 == 0) lbase[r0 * H + h] = lse0;
     }
     if (i1 < C) {
-        float* dst = obase + (r1 * H + h) * D + 2 * t4;
+        const int64_t at = (r1 * H + h) * D + 2 * t4;
 #pragma unroll
-        for (int n = 0; n < ON; ++n)
-            *reinterpret_cast<float2*>(dst + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+        for (int n = 0; n < ON; ++n) {
+            if (to16) *reinterpret_cast<uint32_t*>(static_cast<uint16_t*>(a.out16) + at + n * 8) = pack_out16(o[n][2] * inv1, o[n][3] * inv1, a.out16_bf16);
+            else *reinterpret_cast<float2*>(obase + at + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+        }
         if (t4 == 0) lbase[r1 * H + h] = lse1;
     }
 }

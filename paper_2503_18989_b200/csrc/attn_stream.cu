@@ -349,16 +349,29 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, int n_sub, co
     float* obase; float* lbase; int64_t r0, r1;
     if (item.part < 0) { obase = a.out; lbase = a.lse; r0 = row_base + i0; r1 = row_base + i1; }
     else { obase = a.part_out; lbase = a.part_lse; r0 = item.part + i0; r1 = item.part + i1; }
+    const bool to16 = item.part < 0 && a.out16 != nullptr;      // final rows in the 16-bit output type
     if (i0 < C) {
-        float* dst = obase + (r0 * H + hq0) * D + 2 * t4;
+        const int64_t at = (r0 * H + hq0) * D + 2 * t4;
+        if (to16) {
 #pragma unroll
-        for (int n = 0; n < ON; ++n) *reinterpret_cast<float2*>(dst + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+            for (int n = 0; n < ON; ++n)
+                *reinterpret_cast<uint32_t*>(static_cast<uint16_t*>(a.out16) + at + n * 8) = pack_out16(o[n][0] * inv0, o[n][1] * inv0, a.out16_bf16);
+        } else {
+#pragma unroll
+            for (int n = 0; n < ON; ++n) *reinterpret_cast<float2*>(obase + at + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+        }
         if (t4 == 0) lbase[r0 * H + hq0] = lse0;
     }
     if (i1 < C) {
-        float* dst = obase + (r1 * H + hq1) * D + 2 * t4;
+        const int64_t at = (r1 * H + hq1) * D + 2 * t4;
+        if (to16) {
 #pragma unroll
-        for (int n = 0; n < ON; ++n) *reinterpret_cast<float2*>(dst + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+            for (int n = 0; n < ON; ++n)
+                *reinterpret_cast<uint32_t*>(static_cast<uint16_t*>(a.out16) + at + n * 8) = pack_out16(o[n][2] * inv1, o[n][3] * inv1, a.out16_bf16);
+        } else {
+#pragma unroll
+            for (int n = 0; n < ON; ++n) *reinterpret_cast<float2*>(obase + at + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+        }
         if (t4 == 0) lbase[r1 * H + hq1] = lse1;
     }
 }

@@ -633,9 +633,26 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
                         else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
                         float* dst = obase + (orow * H + u.h) * kD;
-                        // a thread stores its whole row; 32-byte stores fill a sector each (half as many sector writes as
-                        // 16-byte ones, and the sector rate is what bounds this part)
-                        if (wide_stores) {
+                        if (u.part < 0 && a.out16 != nullptr) {
+                            // final rows in the 16-bit output type: 256 bytes per row, eight 32-byte stores
+                            uint16_t* dst16 = static_cast<uint16_t*>(a.out16) + (orow * H + u.h) * kD;
+                            const bool wide16 = (reinterpret_cast<uintptr_t>(a.out16) & 31) == 0;
+#pragma unroll
+                            for (int k = 0; k < kD; k += 16) {
+                                uint32_t w[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) w[e] = pack_out16(o[k + 2 * e] * inv, o[k + 2 * e + 1] * inv, a.out16_bf16);
+                                if (wide16) {
+                                    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
+                                                 ::"l"(dst16 + k), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+                                } else {
+                                    *reinterpret_cast<uint4*>(dst16 + k) = make_uint4(w[0], w[1], w[2], w[3]);
+                                    *reinterpret_cast<uint4*>(dst16 + k + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                                }
+                            }
+                        } else if (wide_stores) {
+                            // a thread stores its whole row; 32-byte stores fill a sector each (half as many sector writes
+                            // as 16-byte ones, and the sector rate is what bounds this part)
 #pragma unroll
                             for (int k = 0; k < kD; k += 8)
                                 st_global_v8(dst + k, o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv, o[k + 4] * inv,

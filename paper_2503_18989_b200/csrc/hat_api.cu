@@ -428,15 +428,17 @@ int hat_kv_append(const hat_cache_desc* cache, const hat_plan* plan, const void*
     return e == cudaSuccess ? HAT_OK : cuda_fail(e);
 }
 
-int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
-                        const void* v_new, float* out, float* lse, float sm_scale, void* workspace,
-                        size_t workspace_bytes, void* stream) {
+// One attention step; the final rows go to `out` (fp32) or, when out16 is given, to out16 in the cache's 16-bit type.
+static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
+                         const void* v_new, float* out, void* out16, float* lse, float sm_scale, void* workspace,
+                         size_t workspace_bytes, void* stream) {
     int st = check_call(cache, plan);
     if (st != HAT_OK) return st;
     if ((k_new == nullptr) != (v_new == nullptr)) return HAT_ERR_INVALID_ARG;
     if (plan->total_rows == 0) return HAT_OK;
-    if (!q || !out || !lse) return HAT_ERR_INVALID_ARG;
-    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(lse, 16)) return HAT_ERR_INVALID_ARG;
+    const void* dst = out16 ? out16 : static_cast<const void*>(out);
+    if (!q || !dst || !lse) return HAT_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(dst, 16) || !aligned(lse, 16)) return HAT_ERR_INVALID_ARG;
     if (k_new && (!aligned(k_new, 16) || !aligned(v_new, 16))) return HAT_ERR_INVALID_ARG;
     const size_t need = (size_t)plan->info.workspace_bytes;
     if (need > 0) {
@@ -466,6 +468,8 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
     a.cache = view_of(cache);
     a.q = q;
     a.out = out;
+    a.out16 = out16;
+    a.out16_bf16 = plan->dtype == HAT_DTYPE_BF16 ? 1 : 0;
     a.lse = lse;
     a.part_out = static_cast<float*>(workspace);
     const int64_t H = plan->num_heads, d = plan->head_dim;
@@ -502,6 +506,21 @@ int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const
         mark(3, 1);
     }
     return HAT_OK;
+}
+
+
+int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
+                        const void* v_new, float* out, float* lse, float sm_scale, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    if (!out && plan && plan->total_rows > 0) return HAT_ERR_INVALID_ARG;
+    return run_attention(cache, plan, q, k_new, v_new, out, nullptr, lse, sm_scale, workspace, workspace_bytes, stream);
+}
+
+int hat_chunk_attention_out16(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
+                              const void* v_new, void* out16, float* lse, float sm_scale, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+    if (!out16 && plan && plan->total_rows > 0) return HAT_ERR_INVALID_ARG;
+    return run_attention(cache, plan, q, k_new, v_new, nullptr, out16, lse, sm_scale, workspace, workspace_bytes, stream);
 }
 
 int hat_plan_verify_event(const hat_plan* plan, void** event_out) {

@@ -60,7 +60,9 @@ struct AttnArgs {
     DevicePlan  plan;
     CacheView   cache;
     const void* q;
-    float*      out;          // [T][H][d]
+    float*      out;          // [T][H][d]; unused when out16 is set
+    void*       out16;        // [T][H][d] in the cache's 16-bit type, or null: final rows go here instead of `out`
+    int         out16_bf16;   // type of out16: 0 = fp16, 1 = bf16
     float*      lse;          // [T][H]
     float*      part_out;     // [part_rows][H][d]
     float*      part_lse;     // [part_rows][H]
@@ -68,6 +70,16 @@ struct AttnArgs {
     long long   wait_cycles;  // bound of every device-side wait, in SM clock cycles
     int         withhold;     // self test: the tile kernel's producer skips its first V tile so that a wait runs out
 };
+
+#ifdef __CUDACC__
+// Two fp32 values rounded to nearest into one 32-bit word of the 16-bit output type (low half = first value).
+__device__ __forceinline__ uint32_t pack_out16(float lo, float hi, int bf16) {
+    uint32_t w;
+    if (bf16) asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.f16x2.f32 %0, %1, %2;\n" : "=r"(w) : "f"(hi), "f"(lo));
+    return w;
+}
+#endif
 
 }  // namespace hat
 

@@ -9,7 +9,7 @@ template <int D>
 __global__ void __launch_bounds__(128)
 merge_kernel(const MergeRow* __restrict__ rows, int num_rows, int H,
              const float* __restrict__ part_out, const float* __restrict__ part_lse,
-             float* __restrict__ out, float* __restrict__ lse) {
+             float* __restrict__ out, float* __restrict__ lse, void* __restrict__ out16, int out16_bf16) {
     const int lane = threadIdx.x & 31;
     const int64_t unit = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);     // (row, head) pair
     if (unit >= (int64_t)num_rows * H) return;
@@ -44,11 +44,17 @@ merge_kernel(const MergeRow* __restrict__ rows, int num_rows, int H,
             acc[0] += ws * v.x; acc[1] += ws * v.y;
         }
     }
-    float* dst = out + ((int64_t)mr.row * H + h) * D + lane * V;
-    if constexpr (V == 4) {
-        *reinterpret_cast<float4*>(dst) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    const int64_t at = ((int64_t)mr.row * H + h) * D + lane * V;
+    if (out16 != nullptr) {
+        uint16_t* dst = static_cast<uint16_t*>(out16) + at;
+        if constexpr (V == 4)
+            *reinterpret_cast<uint2*>(dst) = make_uint2(pack_out16(acc[0], acc[1], out16_bf16), pack_out16(acc[2], acc[3], out16_bf16));
+        else
+            *reinterpret_cast<uint32_t*>(dst) = pack_out16(acc[0], acc[1], out16_bf16);
+    } else if constexpr (V == 4) {
+        *reinterpret_cast<float4*>(out + at) = make_float4(acc[0], acc[1], acc[2], acc[3]);
     } else {
-        *reinterpret_cast<float2*>(dst) = make_float2(acc[0], acc[1]);
+        *reinterpret_cast<float2*>(out + at) = make_float2(acc[0], acc[1]);
     }
     if (lane == 0) lse[(int64_t)mr.row * H + h] = sum > 0.f ? ms + logf(sum) : -INFINITY;
 }
@@ -61,10 +67,10 @@ cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, int first_r
     const unsigned blocks = (unsigned)((units + 3) / 4);
     if (plan->head_dim == 128)
         merge_kernel<128><<<blocks, 128, 0, stream>>>(plan->dev.merge_rows + first_row, n, H, args.part_out, args.part_lse,
-                                                      args.out, args.lse);
+                                                      args.out, args.lse, args.out16, args.out16_bf16);
     else
         merge_kernel<64><<<blocks, 128, 0, stream>>>(plan->dev.merge_rows + first_row, n, H, args.part_out, args.part_lse,
-                                                     args.out, args.lse);
+                                                     args.out, args.lse, args.out16, args.out16_bf16);
     count_launch();
     return cudaGetLastError();
 }

@@ -57,6 +57,14 @@ class DeviceStep:
     def append(self, stream: int = 0) -> None:
         B.hat_kv_append(self.cache.desc, self.plan, self.k_new, self.v_new, stream)
 
+    def attend16(self, fused_append: bool = True, sm_scale: float = 0.0, stream: int = 0) -> None:
+        """The same step with the output in the cache's 16-bit type (self.out16, allocated on first use)."""
+        if getattr(self, "out16", None) is None:
+            self.out16 = torch.full(self.out.shape, -1, dtype=torch.int16, device=self.out.device)
+        B.hat_chunk_attention_out16(self.cache.desc, self.plan, self.q,
+                                    self.k_new if fused_append else None, self.v_new if fused_append else None,
+                                    self.out16, self.lse, sm_scale, self.workspace, self.workspace_bytes, stream)
+
     def attend(self, fused_append: bool = True, sm_scale: float = 0.0, stream: int = 0) -> None:
         B.hat_chunk_attention(self.cache.desc, self.plan, self.q,
                               self.k_new if fused_append else None, self.v_new if fused_append else None,

@@ -423,3 +423,38 @@ def test_grouped_heads_and_trees_on_the_mma_sync_kernels(cuda_device, which, mon
     monkeypatch.setenv("HAT_STREAM_KERNEL" if which == "stream" else "HAT_PREFILL_KERNEL", "mma")
     sc = _manual("bf16", 2, 128, _GQA_PREFIX, _GQA_CHUNK, 61, q_group=4, tree=True)
     _check_full(sc, cuda_device)
+
+
+# ----------------------------------------------------------------------------
+# output in the cache's 16-bit type
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,group", [("fp16", 128, 1), ("bf16", 128, 2), ("fp16", 64, 1), ("bf16", 64, 4)])
+def test_sixteen_bit_output(cuda_device, dtype, d, group, monkeypatch):
+    """hat_chunk_attention_out16: every kernel's final rows (streaming, tile, and rows merged from key ranges)
+    equal the fp32 entry point's rows rounded to nearest, bit for bit where no fp32 value sits on a rounding
+    boundary, and lie within the tolerance plus half a unit in the last place of the oracle's value."""
+    from paper_2503_18989_b200 import runner
+    monkeypatch.setenv("HAT_PREFILL_SPLIT_LEN", "256")           # some tile rows go through the merge kernel too
+    sc = _manual(dtype, 2, d, _GQA_PREFIX + [9000], _GQA_CHUNK + [5], 71, q_group=group)
+    st = sc.steps[0]
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    assert ds.info["num_merge_rows"] > 0
+    ds.attend()
+    o32, l32 = ds.results()
+    ds.attend16(fused_append=False)
+    import torch
+    torch.cuda.synchronize()
+    bits = ds.out16.cpu().numpy().view(np.uint16)
+    got = W.bits_to_f64(bits, dtype)
+    assert np.array_equal(ds.lse.cpu().numpy(), l32), "lse must not depend on the output type"
+    want_bits = W.f32_to_bits(o32, dtype)
+    exact = np.mean(bits == want_bits)
+    assert exact > 0.999, f"only {exact:.4f} of the 16-bit outputs equal the rounded fp32 outputs"
+    assert np.max(np.abs(bits.astype(np.int32) - want_bits.astype(np.int32))[np.isfinite(got)]) <= 1
+    kp, vp, want = oracle_replay(sc)
+    ref = want[0][0]
+    ulp_half = np.abs(ref) * (2.0 ** -11 if dtype == "fp16" else 2.0 ** -8)
+    err = np.abs(got - ref)
+    from common import ABS_TOL
+    assert np.all(err <= ABS_TOL + ulp_half), f"max excess {np.max(err - ulp_half):.3e}"
