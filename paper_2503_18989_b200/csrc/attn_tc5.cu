@@ -702,7 +702,8 @@ bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t
                                H, stride_page, stride_token, stride_head);
 }
 
-cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
+cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit,
+                            bool reset_counter) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     CUtensorMap mq, mk, mv;
     if (!encode_q_map(&mq, bf16, args.q, plan->total_rows, plan->num_heads) ||
@@ -714,9 +715,12 @@ cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStre
     // one CTA per SM draws (item, head) units from a counter that is cleared on the stream first
     const int total_units = (int)plan->prefill_items.size() * plan->num_heads;
     int32_t* counter = plan->dev.status + 1;
-    cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(int32_t), stream);
+    cudaError_t e = cudaSuccess;
+    if (reset_counter) e = cudaMemsetAsync(counter, 0, sizeof(int32_t), stream);
     if (e != cudaSuccess) return e;
-    const dim3 grid((unsigned)std::min(total_units, plan->num_sms));
+    int ctas = std::min(total_units, plan->num_sms);
+    if (grid_limit > 0) ctas = std::min(ctas, grid_limit);
+    const dim3 grid((unsigned)ctas);
     if (bf16) {
         e = cudaFuncSetAttribute(attn_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;

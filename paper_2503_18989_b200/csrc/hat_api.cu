@@ -324,6 +324,9 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->timing = nullptr;
     p->num_verify_merge_rows = 0;
     p->ev_verify = nullptr;
+    p->side_sms = 0;
+    p->aux_stream = nullptr;
+    p->ev_fork = p->ev_join = nullptr;
     p->wait_cycles = 2000000000LL;
     p->withhold_next = 0;
     std::memset(&p->info, 0, sizeof p->info);
@@ -384,6 +387,23 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         if (st != HAT_OK) { hat_plan_destroy(p); return st; }
         cudaError_t ee = cudaEventCreateWithFlags(&p->ev_verify, cudaEventDisableTiming);
         if (ee != cudaSuccess) { p->ev_verify = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
+        // Optional throughput mode for a mixed batch on the tcgen05 path (HAT_SIDE_SMS = n > 0): see the launch
+        // sequence.  Off by default: it finishes the whole step sooner but the decode-phase rows later.  The side
+        // stream has the highest priority so that the tile CTAs are placed before the streaming kernel's many small
+        // CTAs fill the SMs.
+        if (!p->verify_items.empty() && !p->prefill_items.empty() && p->info.prefill_kernel == 1) {
+            int side = env_int("HAT_SIDE_SMS", 0);
+            side = std::max(0, std::min(side, p->num_sms - 8));
+            if (side > 0) {
+                int lo = 0, hi = 0;
+                ee = cudaDeviceGetStreamPriorityRange(&lo, &hi);
+                if (ee == cudaSuccess) ee = cudaStreamCreateWithPriority(&p->aux_stream, cudaStreamNonBlocking, hi);
+                if (ee == cudaSuccess) ee = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
+                if (ee == cudaSuccess) ee = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
+                if (ee != cudaSuccess) { hat_plan_destroy(p); return cuda_fail(ee); }
+                p->side_sms = side;
+            }
+        }
     }
     *out = p;
     return HAT_OK;
@@ -409,6 +429,9 @@ int hat_plan_destroy(hat_plan* plan) {
         delete plan->timing;
     }
     if (plan->ev_verify) cudaEventDestroy(plan->ev_verify);
+    if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
+    if (plan->ev_join) cudaEventDestroy(plan->ev_join);
+    if (plan->aux_stream) cudaStreamDestroy(plan->aux_stream);
     if (plan->dev_blob) {
         cudaError_t e = cudaFree(plan->dev_blob);
         if (e != cudaSuccess) st = cuda_fail(e);
@@ -483,6 +506,18 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
     // Decode-phase (draft verification) requests first: their rows are final, and announced through the plan's event,
     // before the prompt chunks of the same batch are computed, so that they are not held back by them.
     const int n_vm = plan->num_verify_merge_rows, n_m = (int)plan->merge_rows.size();
+    // Mixed batch: the tile kernel starts at once on all but side_sms SMs (own stream), the streaming kernel takes the
+    // rest, and when it is done a second tile grid joins on the SMs it frees; both grids draw from one unit counter.
+    const bool side = plan->side_sms > 0;
+    if (side) {
+        if ((e = cudaMemsetAsync(plan->dev.status + 1, 0, sizeof(int32_t), s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(plan->ev_fork, s)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(plan->aux_stream, plan->ev_fork, 0)) != cudaSuccess) return cuda_fail(e);
+        mark(1, 0);
+        e = launch_attn_tc5(plan, a, plan->aux_stream, plan->num_sms - plan->side_sms, /*reset_counter=*/false);
+        if (e == cudaSuccess) e = cudaEventRecord(plan->ev_join, plan->aux_stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     if (!plan->verify_items.empty()) {
         mark(2, 0);
         e = plan->info.stream_kernel == 1 ? launch_attn_stream(plan, a, s)
@@ -492,7 +527,12 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
         mark(2, 1);
     }
     if (plan->ev_verify && (e = cudaEventRecord(plan->ev_verify, s)) != cudaSuccess) return cuda_fail(e);
-    if (!plan->prefill_items.empty()) {
+    if (side) {
+        e = launch_attn_tc5(plan, a, s, plan->side_sms, /*reset_counter=*/false);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, plan->ev_join, 0);
+        if (e != cudaSuccess) return cuda_fail(e);
+        mark(1, 1);
+    } else if (!plan->prefill_items.empty()) {
         mark(1, 0);
         e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
                                            : launch_attn_mma(plan, a, /*verify_class=*/false, s);

@@ -109,6 +109,12 @@ struct hat_plan {
     hat::Timing* timing;        // null unless hat_plan_enable_timing was called
     int num_verify_merge_rows;  // merge rows of streaming-class requests; they come first in merge_rows
     cudaEvent_t ev_verify;      // recorded in every attention call once the streaming-class rows are final
+    // mixed batches: the tile kernel starts on side_sms fewer SMs on a stream of its own while the streaming kernel
+    // (bound by HBM, which far fewer than all SMs saturate) runs on the caller's stream; a second tile grid joins
+    // on the freed SMs
+    int side_sms;
+    cudaStream_t aux_stream;
+    cudaEvent_t ev_fork, ev_join;
     long long wait_cycles;      // bound of device-side waits (default: about a second)
     int withhold_next;          // self test of the bounded waits: applies to the next attention call only
     void* dev_blob;             // one allocation holding every device array
@@ -124,7 +130,9 @@ cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, int first_r
 // tcgen05 tile kernel (head_dim 128): whether a TMA descriptor can be built for this pool layout, and the launcher
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                           int64_t stride_head);
-cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+// grid_limit > 0 caps the number of CTAs; reset_counter = false joins a grid that is already drawing units
+cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit = 0,
+                            bool reset_counter = true);
 // TMA-fed streaming kernel: whether a TMA descriptor can be built for this pool layout, and the launcher
 bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                              int64_t stride_head);

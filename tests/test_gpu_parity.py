@@ -458,3 +458,20 @@ def test_sixteen_bit_output(cuda_device, dtype, d, group, monkeypatch):
     err = np.abs(got - ref)
     from common import ABS_TOL
     assert np.all(err <= ABS_TOL + ulp_half), f"max excess {np.max(err - ulp_half):.3e}"
+
+
+def test_mixed_batch_with_the_tile_kernel_on_a_side_stream(cuda_device, monkeypatch):
+    """Optional throughput mode: the tile kernel starts on all but 56 SMs on a stream of the plan while the streaming
+    kernel runs, and a second tile grid joins on the freed SMs; same results, also when called back to back."""
+    from paper_2503_18989_b200 import runner
+    monkeypatch.setenv("HAT_SIDE_SMS", "56")
+    sc = W.mixed_13b(num_prefill=5, prefill_chunk=384, max_prefill_prefix=3000, num_verify=12, min_verify_prefix=100,
+                     max_verify_prefix=2000, H=4, seed=81)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    for _ in range(3):
+        ds.attend()
+    go, gl = ds.results()
+    kp, vp, want = oracle_replay(sc)
+    assert_parity(go, want[0][0], "side-stream out")
+    assert_parity(gl, want[0][1], "side-stream lse")
