@@ -250,6 +250,9 @@ def main():
     ap.add_argument("--out16", action="store_true",
                     help="device-resident timing through hat_chunk_attention_out16 (output in the cache's 16-bit type); "
                          "the e2e leg keeps the fp32 host entry point")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture the launch set of one step in a CUDA graph and time its replays (for the launch-bound "
+                         "workloads); the per-kernel figures then come from a separate pass of ordinary launches")
     ap.add_argument("--tree", action="store_true",
                     help="token trees instead of linear drafts on the short chunks (spec_verify and mixed_13b only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -326,8 +329,24 @@ def main():
 
     # ---- timed region: exactly K steps, device events, per-kernel events recorded by the library
     K = args.steps
-    for ds in steps:
-        B.hat_plan_enable_timing(ds.plan, K)
+    run_step, launches_per_replay = one_step, 0
+    if args.graph:
+        gstream = torch.cuda.Stream(device=device)
+        gstream.wait_stream(torch.cuda.current_stream(device))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gstream):
+            n0 = B.hat_launch_count()
+            with torch.cuda.graph(graph, stream=gstream):
+                for ds in steps:
+                    (ds.attend16 if args.out16 else ds.attend)(fused_append=True, stream=gstream.cuda_stream)
+            launches_per_replay = B.hat_launch_count() - n0
+        torch.cuda.current_stream(device).wait_stream(gstream)
+        run_step = graph.replay
+        for _ in range(3):
+            run_step()
+    else:
+        for ds in steps:
+            B.hat_plan_enable_timing(ds.plan, K)
     launches0 = B.hat_launch_count()
     barrier(); torch.cuda.synchronize(device)
     t_wall0 = time.time()
@@ -335,7 +354,7 @@ def main():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(K):
-            one_step()
+            run_step()
         e1.record()
         torch.cuda.synchronize(device)
         elapsed_ms = e0.elapsed_time(e1)
@@ -343,16 +362,27 @@ def main():
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         for a, b in evs:
             flush_buf.zero_()                 # evict the KV working set from L2 (not timed)
-            a.record(); one_step(); b.record()
+            a.record(); run_step(); b.record()
         torch.cuda.synchronize(device)
         elapsed_ms = sum(a.elapsed_time(b) for a, b in evs)
     t_wall1 = time.time()
     barrier()
-    launches = B.hat_launch_count() - launches0
+    launches = B.hat_launch_count() - launches0 + launches_per_replay * K
+    Kk = K
+    if args.graph:
+        # per-kernel durations cannot be read from events inside a graph: one more pass of ordinary launches
+        Kk = min(K, 50)
+        for ds in steps:
+            B.hat_plan_enable_timing(ds.plan, Kk)
+        for _ in range(Kk):
+            if flush_l2:
+                flush_buf.zero_()
+            one_step()
+        torch.cuda.synchronize(device)
     kernel_ms = np.zeros(B.HAT_TIMING_SLOTS)
     kernel_calls = np.zeros(B.HAT_TIMING_SLOTS)
     for ds in steps:
-        ms = B.hat_plan_read_timing(ds.plan, K)
+        ms = B.hat_plan_read_timing(ds.plan, Kk)
         kernel_ms += ms.sum(axis=0)
         kernel_calls += (ms > 0).sum(axis=0)
     clocks = sampler.summary(t_wall0, t_wall1)
@@ -436,6 +466,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": sc.name, "requests": int(sc.steps[-1].num_requests), "rows": total["rows"],
                        "heads": int(sc.steps[-1].q.shape[1]), "kv_heads": sc.cache.num_heads,
+                       "launch": "cuda graph replay" if args.graph else "stream launches",
                        "token_trees": bool(args.tree), "out": "16-bit" if args.out16 else "f32", "head_dim": sc.cache.head_dim, "page_size": 16,
                        "calls_per_step": len(sc.steps), "kv_resident_bytes": int(kv_resident),
                        "l2": "flushed between steps" if flush_l2 else "KV working set larger than L2",

@@ -475,3 +475,33 @@ def test_mixed_batch_with_the_tile_kernel_on_a_side_stream(cuda_device, monkeypa
     kp, vp, want = oracle_replay(sc)
     assert_parity(go, want[0][0], "side-stream out")
     assert_parity(gl, want[0][1], "side-stream lse")
+
+
+def test_the_call_can_be_captured_in_a_cuda_graph_and_replayed(cuda_device):
+    """hat_chunk_attention is stream-ordered and neither allocates nor synchronises, so a caller can capture the
+    launch set of a step (append, streaming kernel, merge, tile kernel) once and replay it."""
+    import torch
+    from paper_2503_18989_b200 import runner
+    sc = W.mixed_13b(num_prefill=3, prefill_chunk=300, max_prefill_prefix=5000, num_verify=6, min_verify_prefix=3000,
+                     max_verify_prefix=9000, H=2, seed=91)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert ds.info["num_merge_rows"] > 0
+    side = torch.cuda.Stream(device=cuda_device)
+    side.wait_stream(torch.cuda.current_stream(cuda_device))
+    with torch.cuda.stream(side):
+        ds.attend(stream=side.cuda_stream)                     # warm-up outside the capture
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            ds.attend(stream=side.cuda_stream)
+    torch.cuda.current_stream(cuda_device).wait_stream(side)
+    ds.out.fill_(float("nan")); ds.lse.fill_(float("nan"))
+    for _ in range(3):
+        graph.replay()
+    go, gl = ds.results()
+    kp, vp, want = oracle_replay(sc)
+    assert_parity(go, want[0][0], "graph replay out")
+    assert_parity(gl, want[0][1], "graph replay lse")
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
