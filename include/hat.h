@@ -173,6 +173,28 @@ int hat_kv_append(const hat_cache_desc* cache, const hat_plan* plan,
                   const void* k_new, const void* v_new, void* stream);
 
 /*
+ * Rotary position encoding fused into the append, and the same rotation for
+ * the query rows.  The paper does not spell the position encoding out; its
+ * models (Vicuna-7B/13B, Sec. 4.1) rotate query and key rows by their token
+ * position in every decoder layer before the attention of Sec. 2.1 and cache
+ * the rotated keys.  Chunk row i of request r has position p = prefix_len[r]+i;
+ * pair c of a head (c = 0 .. head_dim/2-1) turns by the angle p * theta^(-2c/head_dim):
+ *     (x_lo, x_hi) -> (x_lo cos - x_hi sin, x_hi cos + x_lo sin)
+ * with (x_lo, x_hi) = (x[c], x[c+head_dim/2]), or (x[2c], x[2c+1]) when
+ * `interleaved` is non-zero.  The rotation is computed in fp32 (the angle in
+ * double) and rounded to the 16-bit type once.
+ *   hat_kv_append_rope   k_new rows are rotated on their way into the K pool, v_new rows are stored as
+ *                        they come: hat_kv_append with the rotation in between.  k_new, v_new as there.
+ *   hat_rope_q           q_out[t][h][:] = rotated q[t][h][:] for all num_q_heads heads; q_out may be q.
+ *                        Both device, [T][num_q_heads][head_dim], 16-byte aligned.
+ *   theta                base of the angles (> 1; 10000 in the models of the paper)
+ * hat_chunk_attention then takes q_out and no k_new/v_new.  Errors: INVALID_ARG, CUDA.
+ */
+int hat_kv_append_rope(const hat_cache_desc* cache, const hat_plan* plan, const void* k_new, const void* v_new,
+                       float theta, int interleaved, void* stream);
+int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, int interleaved, void* stream);
+
+/*
  * Chunk attention (Sec. 2.1 self-attention over the KV cache; Sec. 2.1 / 3.3
  * prompt chunks; Sec. 3.4 draft verification).  For packed row t = cu_chunk[r]+i
  * and head h, with g = prefix_len[r]+i and keys/values j = 0..g read through

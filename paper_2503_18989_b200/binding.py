@@ -32,7 +32,8 @@ DTYPE_CODE = {"fp16": HAT_DTYPE_FP16, "bf16": HAT_DTYPE_BF16}
 EXPORTS = [
     "hat_status_string", "hat_version", "hat_last_cuda_error", "hat_launch_count",
     "hat_plan_create", "hat_plan_get_info", "hat_plan_workspace_bytes", "hat_plan_destroy",
-    "hat_kv_append", "hat_chunk_attention", "hat_chunk_attention_out16", "hat_plan_staging_bytes",
+    "hat_kv_append", "hat_kv_append_rope", "hat_rope_q", "hat_chunk_attention", "hat_chunk_attention_out16",
+    "hat_plan_staging_bytes",
     "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
     "hat_verify_attention_static", "hat_plan_set_wait_limit",
@@ -110,6 +111,10 @@ def lib() -> C.CDLL:
         L.hat_plan_destroy.argtypes = [vp]
         L.hat_kv_append.restype = i32
         L.hat_kv_append.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, vp]
+        L.hat_kv_append_rope.restype = i32
+        L.hat_kv_append_rope.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, C.c_float, i32, vp]
+        L.hat_rope_q.restype = i32
+        L.hat_rope_q.argtypes = [vp, vp, vp, C.c_float, i32, vp]
         L.hat_chunk_attention.restype = i32
         L.hat_chunk_attention.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, vp, vp, vp, C.c_float, vp, sz, vp]
         L.hat_chunk_attention_out16.restype = i32
@@ -252,6 +257,17 @@ def hat_plan_destroy(plan) -> None:
 
 def hat_kv_append(cache: hat_cache_desc, plan, k_new, v_new, stream: int = 0) -> None:
     _check(lib().hat_kv_append(C.byref(cache), _h(plan), _ptr(k_new), _ptr(v_new), stream or None), "hat_kv_append")
+
+
+def hat_kv_append_rope(cache: hat_cache_desc, plan, k_new, v_new, theta: float = 10000.0, interleaved: bool = False,
+                       stream: int = 0) -> None:
+    _check(lib().hat_kv_append_rope(C.byref(cache), _h(plan), _ptr(k_new), _ptr(v_new), C.c_float(theta),
+                                    int(bool(interleaved)), stream or None), "hat_kv_append_rope")
+
+
+def hat_rope_q(plan, q, q_out, theta: float = 10000.0, interleaved: bool = False, stream: int = 0) -> None:
+    _check(lib().hat_rope_q(_h(plan), _ptr(q), _ptr(q_out), C.c_float(theta), int(bool(interleaved)), stream or None),
+           "hat_rope_q")
 
 
 def hat_chunk_attention(cache: hat_cache_desc, plan, q, k_new, v_new, out, lse, sm_scale: float = 0.0,

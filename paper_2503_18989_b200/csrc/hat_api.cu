@@ -451,6 +451,29 @@ int hat_kv_append(const hat_cache_desc* cache, const hat_plan* plan, const void*
     return e == cudaSuccess ? HAT_OK : cuda_fail(e);
 }
 
+int hat_kv_append_rope(const hat_cache_desc* cache, const hat_plan* plan, const void* k_new, const void* v_new,
+                       float theta, int interleaved, void* stream) {
+    int st = check_call(cache, plan);
+    if (st != HAT_OK) return st;
+    if (!(theta > 1.f) || !std::isfinite(theta)) return HAT_ERR_INVALID_ARG;
+    if (plan->total_rows == 0) return HAT_OK;
+    if (!k_new || !v_new || !aligned(k_new, 16) || !aligned(v_new, 16)) return HAT_ERR_INVALID_ARG;
+    const CacheView view = view_of(cache);
+    cudaError_t e = launch_rope(plan, plan->num_kv_heads, theta, interleaved != 0, k_new, nullptr, &view, cache->k_pool,
+                                cache->v_pool, v_new, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? HAT_OK : cuda_fail(e);
+}
+
+int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, int interleaved, void* stream) {
+    if (!plan || plan->host_only) return HAT_ERR_INVALID_ARG;
+    if (!(theta > 1.f) || !std::isfinite(theta)) return HAT_ERR_INVALID_ARG;
+    if (plan->total_rows == 0) return HAT_OK;
+    if (!q || !q_out || !aligned(q, 16) || !aligned(q_out, 16)) return HAT_ERR_INVALID_ARG;
+    cudaError_t e = launch_rope(plan, plan->num_heads, theta, interleaved != 0, q, q_out, nullptr, nullptr, nullptr, nullptr,
+                                static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? HAT_OK : cuda_fail(e);
+}
+
 // One attention step; the final rows go to `out` (fp32) or, when out16 is given, to out16 in the cache's 16-bit type.
 static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
                          const void* v_new, float* out, void* out16, float* lse, float sm_scale, void* workspace,

@@ -82,12 +82,16 @@ def test_positions_follow_the_prefix():
 # ----------------------------------------------------------------------------
 # GPU parity
 # ----------------------------------------------------------------------------
-def _ulp_distance(a_bits, b_bits):
-    """Distance in units of the last place between two arrays of 16-bit float patterns of the same format."""
-    def key(u):
-        u = u.astype(np.int32)
-        return np.where(u & 0x8000, -(u & 0x7FFF), u & 0x7FFF)
-    return np.abs(key(a_bits) - key(b_bits))
+def _assert_rotated(got_bits, want_bits, dtype, what, exact_share):
+    """The fp32 rotation rounded once against the float64 rotation rounded once: equal bits nearly everywhere; where
+    they differ, by one unit in the last place of the value, or, where the two products cancel, by the fp32 rounding of
+    the products (inputs are below 8 in magnitude here: 8 * 2^-19 = 1.5e-5)."""
+    got, want = W.bits_to_f64(got_bits, dtype), W.bits_to_f64(want_bits, dtype)
+    assert np.isfinite(got).all(), what
+    ulp = np.abs(want) * (2.0 ** -10 if dtype == "fp16" else 2.0 ** -7)          # at least one unit in the last place
+    assert np.all(np.abs(got - want) <= ulp + 1.5e-5), (what, float(np.max(np.abs(got - want) - ulp)))
+    share = float(np.mean(got_bits == want_bits))
+    assert share > exact_share, (what, share)
 
 
 @pytest.mark.gpu
@@ -117,18 +121,16 @@ def test_rotating_append_and_query_kernels(cuda_device, dtype, d, interleaved, g
     # (1) the rotated rows
     want_q = R.rope_bits(st.q, pos, dtype, theta, interleaved)
     got_q = q_rot.cpu().numpy().view(np.uint16).reshape(st.q.shape)
-    dist = _ulp_distance(got_q, want_q)
-    assert dist.max() <= 1 and np.mean(dist == 0) > 0.995, (dist.max(), np.mean(dist == 0))
+    _assert_rotated(got_q, want_q, dtype, "rotated q", 0.995)
     want_k = R.rope_bits(st.k_new, pos, dtype, theta, interleaved)
     ref = types.SimpleNamespace(**{**st.__dict__, "k_new": want_k})
     kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
     O.kv_append(sc.cache, kp, vp, ref)
     gk, gv = cache.pools_to_host()
     assert np.array_equal(gv, vp), "V is stored as it comes"
-    dist = _ulp_distance(gk, kp)
-    assert dist.max() <= 1 and np.mean(dist == 0) > 0.9995, (dist.max(), np.mean(dist == 0))
-    touched = gk != sc.k_pool
-    assert not np.any(touched & (kp == sc.k_pool) & (dist > 0)), "a slot outside the chunk was written"
+    written = kp != sc.k_pool                                  # slots the oracle's append changed
+    assert np.array_equal(gk[~written], kp[~written]), "a slot outside the chunk was written"
+    _assert_rotated(gk[written], kp[written], dtype, "rotated K in the pool", 0.995)
 
     # (2) the step on top of it
     B.hat_chunk_attention(cache.desc, ds.plan, q_rot, None, None, ds.out, ds.lse, 0.0, ds.workspace,
