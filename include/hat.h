@@ -34,7 +34,7 @@
 extern "C" {
 #endif
 
-#define HAT_VERSION 100
+#define HAT_VERSION 110   /* 110: hat_batch_desc gained tree_mask; grouped query heads; out16, rope entry points */
 
 /* status codes */
 #define HAT_OK                        0

@@ -28,7 +28,7 @@ def test_library_exports_every_declared_symbol(hat_lib):
 
 
 def test_version_and_status_strings(hat_lib):
-    assert B.hat_version() == 100
+    assert B.hat_version() == 110
     seen = {B.hat_status_string(s) for s in range(0, -8, -1)}
     assert len(seen) == 8 and "unknown status" not in seen
     assert B.hat_status_string(-99) == "unknown status"
