@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <queue>
 
 #include "hat_internal.h"
 
@@ -73,6 +74,64 @@ static int split_len_for(int kv_end, int wanted, int granule) {
     return std::max(wanted, least);
 }
 
+// Key-range length for the tile-class requests of a batch that is too small to fill the persistent tcgen05 kernel.
+// Every candidate length is priced with a small model of that kernel, in SM clock cycles measured on B200: a 128-key
+// step of a 256-row unit (two query tiles) or of a unit of at most 128 rows (two chains share it), the fixed cost of a
+// unit (its Q tiles, refilling the rings, storing its rows), and the merge pass (its launch plus reading every partial
+// row).  Units go to the CTAs longest first, as the kernel draws them.  Returns 0 for "leave every request whole".
+static int pick_prefill_split(const hat_plan* p, int num_sms, int tile_rows, int key_granule) {
+    constexpr int64_t kStepWide = 4000, kStepNarrow = 2200, kUnit = 10000, kMergeLaunch = 5700;
+    constexpr int64_t kMergeBytesPerCycle = 3000;
+    struct Tile { int keys, rows; };
+    std::vector<Tile> tiles;
+    int max_keys = 0;
+    for (int r = 0; r < p->num_requests; ++r) {
+        const int C = p->chunk_len[r];
+        if (C <= 16) continue;
+        for (int row0 = 0; row0 < C; row0 += tile_rows) {
+            const int rows = std::min(tile_rows, C - row0);
+            tiles.push_back(Tile{p->prefix_len[r] + row0 + rows, rows});
+            max_keys = std::max(max_keys, tiles.back().keys);
+        }
+    }
+    const int H = p->num_heads;
+    std::vector<int64_t> units;
+    auto price = [&](int len) -> int64_t {
+        units.clear();
+        int64_t part_rows = 0;
+        for (const Tile& t : tiles) {
+            const int sl = len > 0 ? split_len_for(t.keys, len, key_granule) : t.keys;
+            const int n = ceil_div(t.keys, sl);
+            if (n > 1) part_rows += (int64_t)n * t.rows;
+            for (int s = 0; s < n; ++s) {
+                const int keys = std::min(t.keys, (s + 1) * sl) - s * sl;
+                units.push_back(ceil_div(keys, 128) * (t.rows > 128 ? kStepWide : kStepNarrow) + kUnit);
+            }
+        }
+        std::sort(units.begin(), units.end(), std::greater<int64_t>());
+        std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> sms;
+        for (int i = 0; i < num_sms; ++i) sms.push(0);
+        int64_t makespan = 0;
+        for (int h = 0; h < H; ++h) {
+            for (int64_t u : units) {
+                const int64_t t = sms.top() + u;
+                sms.pop();
+                sms.push(t);
+                makespan = std::max(makespan, t);
+            }
+        }
+        if (part_rows > 0) makespan += kMergeLaunch + part_rows * H * (p->head_dim + 1) * 4 / kMergeBytesPerCycle;
+        return makespan;
+    };
+    int best = 0;
+    int64_t best_cost = price(0);
+    for (int len = 256; len < max_keys; len += (len < 1024 ? 128 : len < 4096 ? 512 : 2048)) {
+        const int64_t c = price(len);
+        if (c < best_cost) { best_cost = c; best = len; }
+    }
+    return best;
+}
+
 static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     const int H = p->num_heads;
     const int R = p->num_requests;
@@ -133,7 +192,9 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     if (psplit < 0) {
         psplit = 0;
         const int64_t want_ctas = (int64_t)num_sms * 2;
-        if (tiles > 0 && tiles * H < want_ctas) {
+        if (tiles > 0 && tiles * H < want_ctas && use_tc5) {
+            psplit = pick_prefill_split(p, num_sms, tile_rows, key_granule);
+        } else if (tiles > 0 && tiles * H < want_ctas) {
             // aim for want_ctas pieces of equal length, not shorter than 256 keys
             const int pieces = ceil_div((int)want_ctas, H);
             psplit = std::max(256, round_up((int)((tile_keys + pieces - 1) / pieces), key_granule));

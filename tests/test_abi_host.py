@@ -157,6 +157,25 @@ def test_schedule_of_prefill_and_mixed_batches(hat_lib):
     assert info["max_splits"] <= 32
 
 
+def test_small_prefill_batches_are_cut_to_fill_one_round_of_the_persistent_kernel(hat_lib):
+    """One request of 256 rows x 32 heads is 32 units for 148 persistent CTAs.  The plan cuts its keys into ranges
+    chosen by a cost model (a step, the fixed cost of a unit, the merge pass): the ranges are multiples of 128 keys,
+    no more than one unit per CTA results, and a short request is left whole because cutting it costs more than it
+    saves."""
+    c = _cache(num_pages=256, H=32)
+    table = [list(range(144))]
+    sms = 148                                                  # what a host-only plan assumes
+    for prefix in (1024, 1792):
+        info = B.hat_plan_get_info(_plan(c, [prefix], [256], table, H=32)).as_dict()
+        L = info["prefill_split_len"]
+        assert info["prefill_kernel"] == 1 and L >= 256 and L % 128 == 0
+        assert info["max_splits"] == -(-(prefix + 256) // L) and info["max_splits"] > 1
+        assert sms // 2 < info["num_prefill_items"] * 32 <= sms
+        assert info["num_merge_rows"] == 256
+    info = B.hat_plan_get_info(_plan(c, [0], [256], table, H=32)).as_dict()
+    assert info["prefill_split_len"] == 0 and info["num_merge_rows"] == 0 and info["workspace_bytes"] == 0
+
+
 def test_grouped_query_heads_change_the_work_but_not_the_cache_traffic(hat_lib):
     c = _cache(num_pages=64, H=4, d=128)
     table = [list(range(40))]
