@@ -153,6 +153,14 @@ int64_t     hat_launch_count(void);
  * Unless HAT_PLAN_HOST_ONLY is set the schedule is uploaded to the current
  * device (one cudaMalloc + one synchronous copy).  A plan can be reused for
  * every layer of the step and must be destroyed with hat_plan_destroy.
+ * One call at a time per plan: the plan owns device state that an attention
+ * call uses while it runs (the work counter of the persistent tile kernel, the
+ * status word, the verify event, the timing recorder).  Calls that take the
+ * same plan must therefore come from one host thread at a time, and the
+ * library keeps them ordered on the device: a call given another stream than
+ * the plan's previous call first makes that stream wait for the previous call
+ * (cudaStreamWaitEvent on an event the plan owns).  To overlap two steps on
+ * one GPU, create two plans.
  * Errors: INVALID_ARG, UNSUPPORTED, OUT_OF_RANGE, CUDA, TOO_LARGE (more than 65535 work items of one class,
  * i.e. key ranges or 256-row tiles, in one batch).  *out is NULL on error.
  */
@@ -209,7 +217,8 @@ int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, in
  *   out, lse         device fp32, 16-byte aligned
  *   sm_scale         <= 0 or NaN selects 1/sqrt(head_dim)
  *   workspace        device, 256-byte aligned, at least hat_plan_workspace_bytes; may be NULL if that is 0.
- *                    Concurrent calls must use different workspaces.
+ *                    Calls on different plans that may overlap must use different workspaces (calls on one
+ *                    plan never overlap, see hat_plan_create).
  * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, CUDA.
  */
 int hat_chunk_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q,
@@ -355,8 +364,14 @@ int hat_ctrl_parallel_draft_steps(const hat_ctrl* ctrl, int device, int draft_le
  * Differences from hat_chunk_attention:
  *   - cu_chunk, prefix_len, chunk_len, block_table are DEVICE arrays (same
  *     shapes and meaning as in hat_batch_desc); the host cannot inspect them,
- *     so they are not validated: page ids are clamped into the pool and rows at
- *     or beyond max_chunk_len are not computed.
+ *     so they are not validated.  Instead every lookup is clamped: a negative
+ *     prefix_len counts as 0, chunk_len is cut to [0, max_chunk_len] (rows at or
+ *     beyond max_chunk_len are not computed and keep what out/lse held),
+ *     prefix_len + chunk_len is cut to max_pages * 16, block-table columns stay
+ *     inside the request's row and page ids inside the pool: wrong descriptor
+ *     values give wrong rows, not reads outside the arrays.  cu_chunk is
+ *     trusted: it addresses q, out and lse.  hat_static_key_range (a pure host
+ *     function) returns the clamped lengths and the key range of each split.
  *   - No append: the chunk's K/V must already be in the cache.
  *   - Every request is cut into HAT_STATIC_SPLITS key ranges of equal length.
  *   - Limit: num_requests * HAT_STATIC_SPLITS * max_chunk_len * heads * (head_dim+1) * 4 bytes
@@ -371,7 +386,7 @@ int hat_ctrl_parallel_draft_steps(const hat_ctrl* ctrl, int device, int draft_le
  *     so nothing has to be cleared, but two calls that overlap in time on the
  *     same GPU (different streams) race on it.  Serialise them.
  * Errors: INVALID_ARG, UNSUPPORTED, TOO_LARGE, CUDA (the cudaError_t is then
- * available from cudaPeekAtLastError, not from hat_last_cuda_error).
+ * available from hat_last_cuda_error on the calling thread).
  */
 #define HAT_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 #define HAT_STATIC_SPLITS 8
@@ -381,6 +396,12 @@ int hat_verify_attention_static(const hat_cache_desc* cache, int num_requests, i
                                 const int32_t* chunk_len, const int32_t* block_table,    /* device */
                                 const void* q, float* out, float* lse,                   /* device */
                                 float sm_scale, void* stream);
+/* Host only, no CUDA call: what split `split` (0 .. HAT_STATIC_SPLITS-1) of a request with these (unvalidated)
+ * lengths computes in hat_verify_attention_static: the clamped prefix, the rows computed and the keys
+ * [kv_begin, kv_end) of the split.  Null outputs are skipped.  INVALID_ARG for max_chunk_len outside 1..16,
+ * max_pages <= 0 or a split outside the range.  (No counterpart in the paper.) */
+int hat_static_key_range(int prefix_len, int chunk_len, int max_chunk_len, int max_pages, int split,
+                         int* prefix, int* rows, int* kv_begin, int* kv_end);
 
 #ifdef __cplusplus
 }

@@ -10,7 +10,8 @@ Eq. 2 updates the grid point nearest to mu^t; g is linear between observed point
 them, is constant with one observed point and 0 with none; the first observation of a moving average is taken as it
 is; Eq. 3 is answered with the smallest integer X in [x_min, x_max] whose upload time reaches the right-hand side.
 
-Pins (tests/test_ctrl.py): the closed form of an exponential moving average, exact reproduction of a linear g,
+Pins (tests/test_ctrl.py): the closed form of an exponential moving average (of mu, and of the per-device
+quantities with two different observations), exact reproduction of a linear g,
 the closed-form root of Eq. 3 for constant and for linear g, Eq. 6 evaluated by hand.
 """
 import math

@@ -8,10 +8,10 @@
  *
  * What it defines (fp64 throughout; 16-bit inputs are widened exactly):
  *
- *   hat_oracle_kv_append        the KV cache store of Sec. 2.1 ("KV cache ...
- *                               store precomputed keys and values"), addressed
- *                               through a block table ("page attention",
- *                               Sec. 4.1): logical token p of request r lives
+ *   hat_oracle_kv_append        the KV cache store of Sec. 2.1 (KV cache),
+ *                               addressed through a block table (the paged
+ *                               attention named in Sec. 4.1): logical token p
+ *                               of request r lives
  *                               at page block_table[r][p / page_size], slot
  *                               p % page_size.
  *   hat_oracle_attention_rows   scaled dot-product attention (Sec. 2.1, the
@@ -20,10 +20,9 @@
  *                               all cached tokens of its request plus the
  *                               chunk's own tokens up to and including itself.
  *                               This one mask covers both a prompt chunk
- *                               (Sec. 2.1 "chunks are processed across multiple
- *                               inference steps"; Sec. 3.3) and a draft
+ *                               (Sec. 2.1 Batched Inference; Sec. 3.3) and a draft
  *                               sequence verified in a single inference step
- *                               (Sec. 2.1 "Speculative Decoding"; Sec. 3.4).
+ *                               (Sec. 2.1 Speculative Decoding; Sec. 3.4).
  *   hat_oracle_chunk_attention  the same for every (row, head) of a batch.
  *
  *   Two extensions beyond the paper's own models, both optional:

@@ -4,8 +4,8 @@ TEST INFRASTRUCTURE ONLY: shares no code with the CUDA library; only the tests l
 
 The paper does not spell out the position encoding: its models are Vicuna-7B/13B (Sec. 4.1), whose decoder layers
 rotate the query and key rows by their token position before the attention module of Sec. 2.1, and the key rows are
-cached after that rotation ("KV cache ... store precomputed keys and values", Sec. 2.1).  This file is that rotation
-written out in float64, followed by ONE rounding to the 16-bit storage type:
+cached after that rotation (Sec. 2.1, KV cache).  This file is that rotation written out in float64, followed by ONE
+rounding to the 16-bit storage type:
 
     position of chunk row i of request r:   p = prefix_len[r] + i
     angle of pair c (c = 0 .. d/2 - 1):     a = p * theta ** (-2 c / d)
@@ -20,7 +20,16 @@ from __future__ import annotations
 
 import numpy as np
 
-from paper_2503_18989_b200 import workloads as W
+
+def bits_to_f64(bits: np.ndarray, dtype: str) -> np.ndarray:
+    """fp16 / bf16 bit patterns widened exactly to float64 (the oracle's own decoder)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    if dtype == "fp16":
+        return bits.view(np.float16).astype(np.float64)
+    if dtype != "bf16":
+        raise ValueError(dtype)
+    # a bf16 pattern is the upper half of the float32 with the same value
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
 def round_to_bits(x: np.ndarray, dtype: str) -> np.ndarray:
@@ -73,5 +82,5 @@ def rotate(x: np.ndarray, pos: np.ndarray, theta: float = 10000.0, interleaved: 
 def rope_bits(bits: np.ndarray, pos: np.ndarray, dtype: str, theta: float = 10000.0,
               interleaved: bool = False) -> np.ndarray:
     """16-bit rows in, rotated 16-bit rows out (one rounding)."""
-    x = W.bits_to_f64(bits, dtype).reshape(bits.shape)
+    x = bits_to_f64(bits, dtype).reshape(bits.shape)
     return round_to_bits(rotate(x, pos, theta, interleaved), dtype)

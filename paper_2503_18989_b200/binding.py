@@ -36,7 +36,7 @@ EXPORTS = [
     "hat_plan_staging_bytes",
     "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
-    "hat_verify_attention_static", "hat_plan_set_wait_limit",
+    "hat_verify_attention_static", "hat_static_key_range", "hat_plan_set_wait_limit",
     "hat_plan_verify_event", "hat_plan_wait_verify",
     "hat_ctrl_create", "hat_ctrl_destroy", "hat_ctrl_observe", "hat_ctrl_mu", "hat_ctrl_predict",
     "hat_ctrl_device_observe", "hat_ctrl_device_state", "hat_ctrl_chunk_size", "hat_ctrl_parallel_draft_steps",
@@ -149,6 +149,8 @@ def lib() -> C.CDLL:
         L.hat_verify_attention_static.restype = i32
         L.hat_verify_attention_static.argtypes = [C.POINTER(hat_cache_desc), i32, i32, i32, i32, vp, vp, vp, vp,
                                                   vp, vp, vp, C.c_float, vp]
+        L.hat_static_key_range.restype = i32
+        L.hat_static_key_range.argtypes = [i32, i32, i32, i32, i32] + [C.POINTER(i32)] * 4
         _lib = L
     return _lib
 
@@ -319,6 +321,14 @@ def hat_verify_attention_static(cache: hat_cache_desc, num_requests: int, num_q_
                                              int(max_chunk_len), int(max_pages), _ptr(cu_chunk), _ptr(prefix_len),
                                              _ptr(chunk_len), _ptr(block_table), _ptr(q), _ptr(out), _ptr(lse),
                                              float(sm_scale), stream or None), "hat_verify_attention_static")
+
+
+def hat_static_key_range(prefix_len: int, chunk_len: int, max_chunk_len: int, max_pages: int, split: int):
+    """(prefix, rows, kv_begin, kv_end) of one split of hat_verify_attention_static; host only."""
+    o = [C.c_int32() for _ in range(4)]
+    _check(lib().hat_static_key_range(int(prefix_len), int(chunk_len), int(max_chunk_len), int(max_pages), int(split),
+                                      *[C.byref(x) for x in o]), "hat_static_key_range")
+    return tuple(x.value for x in o)
 
 
 def hat_plan_set_wait_limit(plan, cycles: int = 0, withhold_next_call: bool = False) -> None:

@@ -92,12 +92,11 @@ __global__ void __launch_bounds__(128) static_stream_kernel(StaticArgs a) {
     const uint32_t sbase = s_u32(smem);
     const int h = blockIdx.x, r = blockIdx.y / kSplits, sp = blockIdx.y % kSplits;
     const int H = a.num_heads;
-    const int P = a.prefix_len[r];
-    const int C = min(a.chunk_len[r], a.max_rows);
+    // lengths come from device memory nobody validated: clamp them so that no lookup leaves the block table
+    const hat::StaticRange rg = hat::static_key_range(a.prefix_len[r], a.chunk_len[r], a.max_rows, a.max_pages, sp);
+    const int P = rg.prefix, C = rg.rows;
     if (C <= 0) return;
-    const int N = P + C;
-    const int per = ((N + kSplits - 1) / kSplits + 15) / 16 * 16;          // keys per range, whole pages
-    const int kv_begin = sp * per, kv_end = min(N, kv_begin + per);
+    const int kv_begin = rg.kv_begin, kv_end = rg.kv_end;
     const int row_base = a.cu_chunk[r];
     const int32_t* __restrict__ table = a.block_table + (int64_t)r * a.max_pages;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
@@ -116,8 +115,8 @@ __global__ void __launch_bounds__(128) static_stream_kernel(StaticArgs a) {
     auto issue = [&](int ti, int slot) {
         const int kb = kv_begin + ti * 16;
         const uint32_t kdst = ring + slot * (2 * PAGE_BYTES), vdst = kdst + PAGE_BYTES;
-        int page = __ldg(table + kb / 16);
-        page = min(max(page, 0), a.num_pages - 1);                          // never leave the pool
+        int page = __ldg(table + min(kb / 16, a.max_pages - 1));            // never leave the request's table row
+        page = min(max(page, 0), a.num_pages - 1);                          // nor the pool
 #pragma unroll
         for (int idx = lane; idx < 16 * CH; idx += 32) {
             const int row = idx / CH, c = idx % CH;
@@ -300,7 +299,7 @@ __global__ void __launch_bounds__(128) static_merge_kernel(StaticArgs a, int num
     const int h = (int)(unit % H);
     const int i = (int)((unit / H) % a.max_rows);
     const int r = (int)(unit / ((int64_t)H * a.max_rows));
-    if (i >= min(a.chunk_len[r], a.max_rows)) return;
+    if (i >= hat::static_key_range(a.prefix_len[r], a.chunk_len[r], a.max_rows, a.max_pages, 0).rows) return;
     float my = -INFINITY;
     if (lane < kSplits) my = a.part_lse[(((int64_t)r * kSplits + lane) * a.max_rows + i) * H + h];
     float mx = my;
@@ -371,11 +370,11 @@ extern "C" int hat_verify_attention_static(const hat_cache_desc* cache, int num_
     // first call on a device: resolve the device address of the scratch array (no allocation)
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HAT_ERR_CUDA;
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) { hat::set_last_cuda_error((int)e); return HAT_ERR_CUDA; }
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_scratch);
-        if (e != cudaSuccess || !p) return HAT_ERR_CUDA;
+        if (e != cudaSuccess || !p) { hat::set_last_cuda_error((int)e); return HAT_ERR_CUDA; }
         g_scratch_addr[dev] = p;
     }
     if (!(sm_scale > 0.f) || !std::isfinite(sm_scale)) sm_scale = 1.0f / std::sqrt((float)d);
@@ -393,5 +392,18 @@ extern "C" int hat_verify_attention_static(const hat_cache_desc* cache, int num_
     const bool bf16 = cache->dtype == HAT_DTYPE_BF16;
     if (d == 128) e = bf16 ? launch_static<true, 128>(a, num_requests, s) : launch_static<false, 128>(a, num_requests, s);
     else e = bf16 ? launch_static<true, 64>(a, num_requests, s) : launch_static<false, 64>(a, num_requests, s);
+    if (e != cudaSuccess) hat::set_last_cuda_error((int)e);
     return e == cudaSuccess ? HAT_OK : HAT_ERR_CUDA;
+}
+
+extern "C" int hat_static_key_range(int prefix_len, int chunk_len, int max_chunk_len, int max_pages, int split,
+                                    int* prefix, int* rows, int* kv_begin, int* kv_end) {
+    if (max_chunk_len < 1 || max_chunk_len > 16 || max_pages <= 0 || split < 0 || split >= HAT_STATIC_SPLITS)
+        return HAT_ERR_INVALID_ARG;
+    const hat::StaticRange rg = hat::static_key_range(prefix_len, chunk_len, max_chunk_len, max_pages, split);
+    if (prefix) *prefix = rg.prefix;
+    if (rows) *rows = rg.rows;
+    if (kv_begin) *kv_begin = rg.kv_begin;
+    if (kv_end) *kv_end = rg.kv_end;
+    return HAT_OK;
 }

@@ -16,6 +16,7 @@ static thread_local int g_last_cuda_error = 0;
 static std::atomic<int64_t> g_launches{0};
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
 static int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
@@ -385,6 +386,9 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->timing = nullptr;
     p->num_verify_merge_rows = 0;
     p->ev_verify = nullptr;
+    p->ev_done = nullptr;
+    p->last_stream = nullptr;
+    p->has_last = false;
     p->side_sms = 0;
     p->aux_stream = nullptr;
     p->ev_fork = p->ev_join = nullptr;
@@ -448,6 +452,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         if (st != HAT_OK) { hat_plan_destroy(p); return st; }
         cudaError_t ee = cudaEventCreateWithFlags(&p->ev_verify, cudaEventDisableTiming);
         if (ee != cudaSuccess) { p->ev_verify = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
+        ee = cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming);
+        if (ee != cudaSuccess) { p->ev_done = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
         // Optional throughput mode for a mixed batch on the tcgen05 path (HAT_SIDE_SMS = n > 0): see the launch
         // sequence.  Off by default: it finishes the whole step sooner but the decode-phase rows later.  The side
         // stream has the highest priority so that the tile CTAs are placed before the streaming kernel's many small
@@ -490,6 +496,7 @@ int hat_plan_destroy(hat_plan* plan) {
         delete plan->timing;
     }
     if (plan->ev_verify) cudaEventDestroy(plan->ev_verify);
+    if (plan->ev_done) cudaEventDestroy(plan->ev_done);
     if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
     if (plan->ev_join) cudaEventDestroy(plan->ev_join);
     if (plan->aux_stream) cudaStreamDestroy(plan->aux_stream);
@@ -556,6 +563,15 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
+    // The plan's device state (unit counter, status word) serves one call at a time: a call on another stream than the
+    // previous one is ordered behind it.
+    hat_plan* mplan = const_cast<hat_plan*>(plan);
+    if (plan->has_last && plan->last_stream != s && (e = cudaStreamWaitEvent(s, plan->ev_done, 0)) != cudaSuccess)
+        return cuda_fail(e);
+    struct Done {
+        hat_plan* p; cudaStream_t s;
+        ~Done() { if (p->ev_done && cudaEventRecord(p->ev_done, s) == cudaSuccess) { p->last_stream = s; p->has_last = true; } }
+    } done{mplan, s};
     // optional event recorder: a start and an end event per slot (append, tile, streaming, merge)
     Timing* tm = plan->timing;
     int call = -1;

@@ -71,6 +71,28 @@ struct AttnArgs {
     int         withhold;     // self test: the tile kernel's producer skips its first V tile so that a wait runs out
 };
 
+// Key range of one split of the allocation-free streaming entry point, from lengths that nobody validated (they are
+// read from device memory).  A negative prefix counts as 0, the chunk is cut to [0, max_rows], and prefix + chunk is
+// cut to the max_pages * 16 tokens one row of the block table can address: wrong lengths then give wrong rows, never a
+// lookup outside the table.  Ranges are whole pages, HAT_STATIC_SPLITS of equal length; trailing ranges may be empty.
+struct StaticRange { int prefix, rows, kv_begin, kv_end; };
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline StaticRange static_key_range(int prefix_len, int chunk_len, int max_rows, int max_pages, int split) {
+    const long long cap = (long long)max_pages * kPageSize;
+    long long P = prefix_len < 0 ? 0 : prefix_len;
+    long long C = chunk_len < 0 ? 0 : (chunk_len > max_rows ? max_rows : chunk_len);
+    if (P > cap) P = cap;
+    if (P + C > cap) C = cap - P;
+    const long long N = P + C;
+    const long long per = ((N + HAT_STATIC_SPLITS - 1) / HAT_STATIC_SPLITS + kPageSize - 1) / kPageSize * kPageSize;
+    long long b = (long long)split * per, e = b + per;
+    if (b > N) b = N;
+    if (e > N) e = N;
+    return StaticRange{(int)P, (int)C, (int)b, (int)e};
+}
+
 #ifdef __CUDACC__
 // Two fp32 values rounded to nearest into one 32-bit word of the 16-bit output type (low half = first value).
 __device__ __forceinline__ uint32_t pack_out16(float lo, float hi, int bf16) {
@@ -109,6 +131,9 @@ struct hat_plan {
     hat::Timing* timing;        // null unless hat_plan_enable_timing was called
     int num_verify_merge_rows;  // merge rows of streaming-class requests; they come first in merge_rows
     cudaEvent_t ev_verify;      // recorded in every attention call once the streaming-class rows are final
+    cudaEvent_t ev_done;        // recorded at the end of every attention call: the next call on another stream waits for it
+    cudaStream_t last_stream;   // stream of the previous attention call
+    bool has_last;
     // mixed batches: the tile kernel starts on side_sms fewer SMs on a stream of its own while the streaming kernel
     // (bound by HBM, which far fewer than all SMs saturate) runs on the caller's stream; a second tile grid joins
     // on the freed SMs
@@ -142,4 +167,5 @@ bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int6
                              int64_t stride_head);
 cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
 void count_launch(int n = 1);
+void set_last_cuda_error(int e);   // what hat_last_cuda_error() returns on this thread
 }  // namespace hat

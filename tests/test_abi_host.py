@@ -201,3 +201,38 @@ def test_batches_beyond_the_launch_limits_are_rejected(hat_lib):
     table = np.arange(n, dtype=np.int32)[:, None]
     assert _status(_plan, c, np.zeros(n, np.int32), np.ones(n, np.int32), table, H=1) == B.HAT_ERR_TOO_LARGE
     assert _status(_plan, c, np.zeros(60000, np.int32), np.ones(60000, np.int32), table[:60000], H=1) == B.HAT_OK
+
+
+def test_static_entry_point_clamps_unvalidated_lengths(hat_lib):
+    """hat_verify_attention_static reads its lengths from device memory nobody checked; the helper that turns them
+    into key ranges must keep every block-table lookup inside the request's row whatever they hold."""
+    S = B.HAT_STATIC_SPLITS
+    # a sane request: the ranges tile [0, P + C) in whole pages, in order
+    ranges = [B.hat_static_key_range(1000, 5, 8, 100, sp) for sp in range(S)]
+    assert all(r[0] == 1000 and r[1] == 5 for r in ranges)
+    assert ranges[0][2] == 0 and ranges[-1][3] == 1005
+    for a, b in zip(ranges, ranges[1:]):
+        assert a[3] == b[2] and a[2] % 16 == 0 and a[2] <= a[3]
+    per = ((1005 + S - 1) // S + 15) // 16 * 16
+    assert ranges[0][3] == per
+    # overstated, negative and oversized lengths (nothing here is sent to a GPU)
+    rng = np.random.default_rng(7)
+    cases = [(10**9, 16, 16, 5), (-5, 3, 8, 4), (0, 10**6, 16, 1), (79, 16, 16, 5), (80, 1, 16, 5), (2**31 - 1, 2**31 - 1, 16, 3)]
+    cases += [(int(rng.integers(-100, 5000)), int(rng.integers(-5, 40)), int(rng.integers(1, 17)), int(rng.integers(1, 64)))
+              for _ in range(200)]
+    for P, Cl, max_rows, max_pages in cases:
+        cover = 0
+        for sp in range(S):
+            prefix, rows, b, e = B.hat_static_key_range(P, Cl, max_rows, max_pages, sp)
+            assert 0 <= prefix and 0 <= rows <= max_rows and prefix + rows <= max_pages * 16
+            assert 0 <= b <= e <= prefix + rows
+            assert e == b or (e - 1) // 16 <= max_pages - 1          # last page looked up is a column of the table row
+            assert b == cover
+            cover = e
+        assert cover == prefix + rows
+        if 0 <= P and 0 <= Cl <= max_rows and P + Cl <= max_pages * 16:
+            assert (prefix, rows) == (P, Cl)                          # valid lengths pass through unchanged
+    with pytest.raises(B.HatError):
+        B.hat_static_key_range(10, 2, 17, 4, 0)
+    with pytest.raises(B.HatError):
+        B.hat_static_key_range(10, 2, 8, 4, S)

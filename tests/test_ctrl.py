@@ -31,6 +31,32 @@ def test_moving_average_closed_form():
     assert o.mu == 128 and o.predict(128) == 3
 
 
+def test_device_moving_average_closed_form():
+    # Sec. 3.2: the per-device drafting delay and link bandwidths are averaged with the same weight as Eq. 1.
+    # Two DIFFERENT observations: new = alpha * old + (1 - alpha) * x2, for each of the three quantities.
+    a = 0.8
+    o = OracleCtrl(a, 64.0, 256)
+    x1, x2, x3 = (0.010, 6e6, 11e6), (0.030, 9e6, 14e6), (0.020, 5e6, 12e6)
+    o.device_observe(2, *x1)
+    assert o.dev[2] == list(x1)                                  # the first observation is taken as it is
+    o.device_observe(2, *x2)
+    for got, u, v in zip(o.dev[2], x1, x2):
+        assert got == pytest.approx(a * u + (1 - a) * v, rel=1e-15)
+    assert o.dev[2][0] == pytest.approx(0.014, rel=1e-12)         # 0.8 * 10 ms + 0.2 * 30 ms, by hand
+    assert o.dev[2][1] == pytest.approx(6.6e6, rel=1e-12)
+    assert o.dev[2][2] == pytest.approx(11.6e6, rel=1e-12)
+    o.device_observe(2, *x3)
+    for got, u, v, w in zip(o.dev[2], x1, x2, x3):
+        assert got == pytest.approx(a * a * u + a * (1 - a) * v + (1 - a) * w, rel=1e-15)
+    assert 5 not in o.dev                                         # other devices untouched
+    o = OracleCtrl(0.0, 64.0, 256)                                # alpha = 0: the latest observation
+    o.device_observe(0, *x1); o.device_observe(0, *x2)
+    assert o.dev[0] == list(x2)
+    o = OracleCtrl(1.0, 64.0, 256)                                # alpha = 1: frozen at the first
+    o.device_observe(0, *x1); o.device_observe(0, *x2)
+    assert o.dev[0] == list(x1)
+
+
 def test_linear_delay_is_reproduced_and_extrapolated():
     # two observed grid points of g(x) = 2e-3 + 1e-5 x (alpha = 0: mu^t = mu_hat^t) define the whole line
     ga, gb = 2e-3, 1e-5

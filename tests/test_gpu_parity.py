@@ -505,3 +505,22 @@ def test_the_call_can_be_captured_in_a_cuda_graph_and_replayed(cuda_device):
     assert_parity(gl, want[0][1], "graph replay lse")
     gk, gv = cache.pools_to_host()
     assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+
+
+def test_calls_on_one_plan_from_two_streams_are_kept_in_order(cuda_device):
+    """A plan serves one call at a time (its unit counter and status word are shared): calls handed different
+    streams are ordered by the library itself, so alternating streams without any synchronisation is still correct."""
+    import torch
+    from paper_2503_18989_b200 import runner
+    sc = W.ragged_prefill(num_requests=6, max_prefix=1024, H=4, seed=77)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    s1, s2 = torch.cuda.Stream(cuda_device), torch.cuda.Stream(cuda_device)
+    torch.cuda.synchronize()
+    for it in range(6):
+        ds.attend(fused_append=True, stream=(s1 if it % 2 == 0 else s2).cuda_stream)
+    out, lse = ds.results()
+    _, _, want = oracle_replay(sc)
+    assert_parity(out, want[0][0], "two streams out")
+    assert_parity(lse, want[0][1], "two streams lse")
+    ds.close()
