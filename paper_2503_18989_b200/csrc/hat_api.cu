@@ -133,7 +133,10 @@ static int pick_prefill_split(const hat_plan* p, int num_sms, int tile_rows, int
     return best;
 }
 
-static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
+// tile_kernel: 0 = mma.sync, 1 = tcgen05 with two query tiles per CTA, 3 = tcgen05 by pairs of CTAs (cta_group::2) with a
+// ring of three score buffers; both tcgen05 kernels take 256-row units
+static void schedule(hat_plan* p, int num_sms, int tile_kernel) {
+    const bool use_tc5 = tile_kernel != 0;
     const int H = p->num_heads;
     const int R = p->num_requests;
     hat_plan_info& info = p->info;
@@ -143,7 +146,7 @@ static void schedule(hat_plan* p, int num_sms, bool use_tc5) {
     const int tile_rows = use_tc5 ? 256 : 64;
     const int key_granule = use_tc5 ? 128 : 64;
     info.prefill_tile_rows = tile_rows;
-    info.prefill_kernel = use_tc5 ? 1 : 0;
+    info.prefill_kernel = tile_kernel;
 
     // ---- streaming (verify-class) requests: fixed-length key ranges, shortened until the SMs are covered.
     // A CTA of the streaming kernel serves one K/V head and 16 (row, query head of the group) pairs.
@@ -431,7 +434,10 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_kv_heads, cache->stride_page,
                                        cache->stride_token, cache->stride_head);
     p->num_sms = num_sms;
-    schedule(p, num_sms, use_tc5);
+    int tile_kernel = use_tc5 ? 1 : 0;
+    if (const char* k = std::getenv("HAT_PREFILL_KERNEL"))
+        if (use_tc5 && std::strcmp(k, "pair") == 0) tile_kernel = 3;
+    schedule(p, num_sms, tile_kernel);
     // the streaming kernel takes its pages by TMA when a descriptor can be built for the pool layout
     bool stream_tma = true;
     if (const char* k = std::getenv("HAT_STREAM_KERNEL"))
@@ -635,6 +641,7 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
     } else if (!plan->prefill_items.empty()) {
         mark(1, 0);
         e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
+          : plan->info.prefill_kernel == 3 ? launch_attn_pair(plan, a, s)
                                            : launch_attn_mma(plan, a, /*verify_class=*/false, s);
         if (e != cudaSuccess) return cuda_fail(e);
         mark(1, 1);

@@ -162,6 +162,8 @@ bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t
 // grid_limit > 0 caps the number of CTAs; reset_counter = false joins a grid that is already drawing units
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit = 0,
                             bool reset_counter = true);
+// tcgen05 tile kernel with 256-row units processed by clusters of two CTAs (cta_group::2), same layout requirements
+cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
 // TMA-fed streaming kernel: whether a TMA descriptor can be built for this pool layout, and the launcher
 bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                              int64_t stride_head);

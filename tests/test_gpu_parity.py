@@ -268,7 +268,7 @@ def test_bounded_wait_gives_up_and_the_context_stays_usable(cuda_device):
     st = sc.steps[0]
     cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
     ds = runner.DeviceStep(cache, st)
-    assert ds.info["prefill_kernel"] == 1
+    assert ds.info["prefill_kernel"] in (1, 3)
     assert B.hat_last_device_status(ds.plan) == B.HAT_OK
     B.hat_plan_set_wait_limit(ds.plan, 20_000_000, withhold_next_call=True)      # about 10 ms
     ds.attend(fused_append=True)
@@ -311,7 +311,7 @@ def test_key_ranges_that_only_the_second_query_tile_sees(cuda_device, dtype, mon
     from paper_2503_18989_b200 import runner
     cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
     ds = runner.DeviceStep(cache, sc.steps[0])
-    assert ds.info["prefill_kernel"] == 1 and ds.info["prefill_split_len"] == 256 and ds.info["max_splits"] == 5
+    assert ds.info["prefill_kernel"] in (1, 3) and ds.info["prefill_split_len"] == 256 and ds.info["max_splits"] == 5
     _check_full(sc, cuda_device)
 
 
