@@ -144,6 +144,133 @@ def whole_job_value(flops_per_replica_step: int, world: int, ms_per_step: float)
     return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
 
 
+NOMINAL = {"tensor_tflops": 2250.0, "hbm_gbs": 8000.0}      # dense 16-bit tensor peak and HBM3e bandwidth of a B200, nominal
+
+
+def pick_tensor_peak(peaks, peak_kind, timed_seconds, reasons):
+    """Denominator for a tensor-bound kernel: the burst figure when the timed region is well under a second and the
+    sampled clocks show no power cap (a kernel timed alone), else the sustained one (a kernel inside a long loop)."""
+    burst = timed_seconds < 1.0 and "sw_power_cap" not in (reasons or [])
+    key = "bf16_tflops" if burst else "bf16_tflops_sustained"
+    return peaks[key], f"{peak_kind} bf16 {'burst' if burst else 'sustained'}"
+
+
+def kernel_table(total, works, n_calls, kernel_ms, kernel_calls, peaks, tensor_peak):
+    """Per kernel: achieved algorithmic throughput from its mean CUDA-event duration, against every denominator."""
+    avg = np.where(kernel_calls > 0, kernel_ms / np.maximum(kernel_calls, 1), 0.0)   # ms per launch
+    per_launch = {
+        "kv_append": ("hbm", total["append_bytes"] / n_calls),
+        "tile_attention": ("tensor", total["tile_flops"] / max(1, sum(1 for w in works if w["tile_flops"]))),
+        "streaming_attention": ("hbm", total["stream_bytes"] / max(1, sum(1 for w in works if w["stream_bytes"]))),
+        "merge": ("hbm", 0.0),
+    }
+    kernels = {}
+    for i, name in enumerate(SLOT_NAMES):
+        if kernel_calls[i] == 0:
+            continue
+        bound, alg = per_launch[name]
+        sec = avg[i] * 1e-3
+        if bound == "tensor":
+            ach, peak, unit = alg / sec / 1e12, tensor_peak, "TFLOP/s"
+            extra = {"frac_burst": ach / peaks["bf16_tflops"], "frac_sustained": ach / peaks["bf16_tflops_sustained"],
+                     "frac_nominal": ach / NOMINAL["tensor_tflops"]}
+        else:
+            ach, peak, unit = alg / sec / 1e9, peaks["hbm_gbs"], "GB/s"
+            extra = {"frac_nominal": ach / NOMINAL["hbm_gbs"]}
+            if ach > peak:
+                extra["note"] = "above 1: the denominator is a measured COPY (read + write); a read-only stream can exceed it"
+        kernels[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, **extra,
+                         "ms_per_launch": float(avg[i]), "launches": int(kernel_calls[i]),
+                         "share": float(kernel_ms[i] / max(kernel_ms.sum(), 1e-9))}
+    if "tile_attention" in kernels:
+        # the tile kernel against the memory roofline as well (short chunks are HBM-bound)
+        sec = kernels["tile_attention"]["ms_per_launch"] * 1e-3
+        n_tile_calls = max(1, sum(1 for w in works if w["tile_flops"]))
+        kernels["tile_attention"]["algorithmic_bytes"] = int(total["tile_bytes"] / n_tile_calls)
+        kernels["tile_attention"]["hbm_gbs"] = total["tile_bytes"] / n_tile_calls / sec / 1e9
+        kernels["tile_attention"]["hbm_frac"] = kernels["tile_attention"]["hbm_gbs"] / peaks["hbm_gbs"]
+    return kernels
+
+
+def step_bound(total, ms_per_step, peaks, tensor_peak):
+    """Roofline of the whole step: T_roof = max(F / pi, B / beta) over all algorithmic flops and bytes (K/V read once
+    per head, q in, out + lse out, append read + write), measured and nominal peaks."""
+    F = total["flops"]
+    Bt = total["tile_bytes"] + total["stream_bytes"] + total["append_bytes"]
+    t_meas = max(F / (tensor_peak * 1e12), Bt / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    t_nom = max(F / (NOMINAL["tensor_tflops"] * 1e12), Bt / (NOMINAL["hbm_gbs"] * 1e9)) * 1e3
+    return {"flops": int(F), "bytes": int(Bt), "t_roof_ms": t_meas, "step_frac": t_meas / ms_per_step,
+            "t_roof_nominal_ms": t_nom, "step_frac_nominal": t_nom / ms_per_step,
+            "flops_over_peak_ms": F / (tensor_peak * 1e12) * 1e3, "bytes_over_bandwidth_ms": Bt / (peaks["hbm_gbs"] * 1e9) * 1e3}
+
+
+def quick_config(name, device, stream, peaks, peak_kind, K=20, warmup=3, with_oracle=True, samples=96):
+    """One of the named workloads, briefly: K timed steps (L2 flushed where the K/V working set would fit in it),
+    per-kernel roofline figures, and the largest deviation from the CPU oracle on sampled (request, row, head) triples
+    of the last call."""
+    import torch
+    from paper_2503_18989_b200 import binding as B
+    from paper_2503_18989_b200 import runner
+    sc = W.WORKLOADS[name]()
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, device)
+    steps = [runner.DeviceStep(cache, st) for st in sc.steps]
+    works = [step_work(sc.cache, st) for st in sc.steps]
+    total = {k: sum(w[k] for w in works) for k in works[0]}
+    flush_l2 = total["kv_bytes"] / len(sc.steps) < 2 * L2_BYTES
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device) if flush_l2 else None
+
+    def one_step():
+        for ds in steps:
+            ds.attend(fused_append=True, stream=stream)
+    for _ in range(warmup):
+        one_step()
+    torch.cuda.synchronize(device)
+    for ds in steps:
+        B.hat_plan_enable_timing(ds.plan, K)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in evs:
+        if flush_l2:
+            flush_buf.zero_()
+        a.record(); one_step(); b.record()
+    torch.cuda.synchronize(device)
+    elapsed_ms = sum(a.elapsed_time(b) for a, b in evs)
+    kernel_ms = np.zeros(B.HAT_TIMING_SLOTS)
+    kernel_calls = np.zeros(B.HAT_TIMING_SLOTS)
+    for ds in steps:
+        ms = B.hat_plan_read_timing(ds.plan, K)
+        kernel_ms += ms.sum(axis=0)
+        kernel_calls += (ms > 0).sum(axis=0)
+    status = [B.hat_last_device_status(ds.plan, stream) for ds in steps]
+    ms_per_step = elapsed_ms / K
+    tensor_peak, source = pick_tensor_peak(peaks, peak_kind, elapsed_ms * 1e-3, [])
+    res = {"ms_per_step": ms_per_step, "steps": K, "calls_per_step": len(sc.steps), "dtype": sc.cache.dtype,
+           "l2": "flushed between steps" if flush_l2 else "KV working set larger than L2",
+           "value_tflops": total["flops"] / (ms_per_step * 1e-3) / 1e12,
+           "kv_gbs": total["kv_bytes"] / (ms_per_step * 1e-3) / 1e9, "tensor_peak_source": source,
+           "kernels": kernel_table(total, works, len(sc.steps), kernel_ms, kernel_calls, peaks, tensor_peak),
+           "step_roofline": step_bound(total, ms_per_step, peaks, tensor_peak),
+           "device_status_ok": all(s == B.HAT_OK for s in status)}
+    if with_oracle:
+        from oracle import hat_oracle as O
+        st = sc.steps[-1]
+        out, lse = steps[-1].results()
+        kp, vp = cache.pools_to_host()                # the GPU's own pools after the appends (checked bit for bit in tests/)
+        rng = np.random.default_rng(1)
+        live = np.nonzero(st.chunk_len > 0)[0]
+        tri = np.asarray([(r, int(rng.integers(st.chunk_len[r])), int(rng.integers(st.q.shape[1])))
+                          for r in live[rng.integers(len(live), size=samples)]], np.int64)
+        wo, wl = O.attention_rows(sc.cache, kp, vp, st, tri)
+        rows = st.cu_chunk[tri[:, 0]] + tri[:, 1]
+        res["oracle_sample"] = {"triples": int(len(tri)),
+                                "max_abs_out": float(np.abs(out[rows, tri[:, 2]].astype(np.float64) - wo).max()),
+                                "max_abs_lse": float(np.abs(lse[rows, tri[:, 2]].astype(np.float64) - wl).max())}
+    for ds in steps:
+        ds.close()
+    del steps, cache, flush_buf
+    torch.cuda.empty_cache()
+    return res
+
+
 def lookup_traffic(kernel: str, workload: str):
     """DRAM bytes per launch from the committed ncu capture of this kernel on this workload, or None when
     there is none or the kernel source has changed since (profiles/traffic.json records a source hash)."""
@@ -256,8 +383,14 @@ def main():
     ap.add_argument("--tree", action="store_true",
                     help="token trees instead of linear drafts on the short chunks (spec_verify and mixed_13b only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--all-configs", dest="all_configs", action="store_true", default=None,
+                    help="after the main measurement, time the other named workloads briefly (default: on for the default "
+                         "workload on one GPU)")
+    ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
     args = ap.parse_args()
+    if args.all_configs is None:
+        args.all_configs = args.workload == "mixed_13b" and args.gpus == 1 and args.q_group == 1 and not args.tree
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -427,37 +560,24 @@ def main():
         e2e_value = whole_job_value(total["flops"], world, e2e_ms / Ke)
 
         # per-kernel achieved throughput against its roofline
-        avg = np.where(kernel_calls > 0, kernel_ms / np.maximum(kernel_calls, 1), 0.0)   # ms per launch
-        per_launch = {
-            "kv_append": ("hbm", total["append_bytes"] / len(sc.steps)),
-            "tile_attention": ("tensor", total["tile_flops"] / max(1, sum(1 for w in works if w["tile_flops"]))),
-            "streaming_attention": ("hbm", total["stream_bytes"] / max(1, sum(1 for w in works if w["stream_bytes"]))),
-            "merge": ("hbm", 0.0),
-        }
-        tensor_peak = peaks["bf16_tflops_sustained"]
-        kernels = {}
-        for i, name in enumerate(SLOT_NAMES):
-            if kernel_calls[i] == 0:
-                continue
-            bound, alg = per_launch[name]
-            sec = avg[i] * 1e-3
-            if bound == "tensor":
-                ach, peak, unit = alg / sec / 1e12, tensor_peak, "TFLOP/s"
-            else:
-                ach, peak, unit = alg / sec / 1e9, peaks["hbm_gbs"], "GB/s"
-            kernels[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                             "ms_per_launch": float(avg[i]), "launches": int(kernel_calls[i]),
-                             "share": float(kernel_ms[i] / max(kernel_ms.sum(), 1e-9))}
+        timed_seconds = elapsed_ms * 1e-3
+        tensor_peak, tensor_source = pick_tensor_peak(peaks, peak_kind, timed_seconds, clocks.get("reasons"))
+        kernels = kernel_table(total, works, len(sc.steps), kernel_ms, kernel_calls, peaks, tensor_peak)
         dominant = max(kernels, key=lambda n: kernels[n]["share"])
         roof = {k: kernels[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
-        roof.update({"kernel": dominant, "traffic": lookup_traffic(dominant, sc.name), "peak_source": f"{peak_kind} "
-                     + ("bf16 sustained" if roof["bound"] == "tensor" else "HBM copy")})
-        # the tile kernel against the memory roofline as well (short chunks are HBM-bound)
-        if "tile_attention" in kernels:
-            sec = kernels["tile_attention"]["ms_per_launch"] * 1e-3
-            n_tile_calls = max(1, sum(1 for w in works if w["tile_flops"]))
-            kernels["tile_attention"]["hbm_gbs"] = total["tile_bytes"] / n_tile_calls / sec / 1e9
-            kernels["tile_attention"]["hbm_frac"] = kernels["tile_attention"]["hbm_gbs"] / peaks["hbm_gbs"]
+        for k in ("frac_burst", "frac_sustained", "frac_nominal"):
+            if k in kernels[dominant]:
+                roof[k] = kernels[dominant][k]
+        traffic = lookup_traffic(dominant, sc.name)
+        alg_bytes = kernels[dominant].get("algorithmic_bytes")
+        if alg_bytes is None and kernels[dominant]["bound"] == "hbm":
+            alg_bytes = int(kernels[dominant]["achieved"] * 1e9 * kernels[dominant]["ms_per_launch"] * 1e-3)
+        roof.update({"kernel": dominant, "traffic": traffic, "algorithmic_bytes": alg_bytes,
+                     "traffic_over_algorithmic": (traffic / alg_bytes) if (traffic and alg_bytes) else None,
+                     "peak_source": tensor_source if roof["bound"] == "tensor" else f"{peak_kind} HBM copy",
+                     "timed_seconds": timed_seconds,
+                     "ms_per_launch_x_sm_mhz": (kernels[dominant]["ms_per_launch"] * clocks["sm_mhz"])
+                     if clocks.get("sm_mhz") else None})
 
         line = {
             "metric": "chunk_attention_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
@@ -478,6 +598,7 @@ def main():
             "roofline": roof,
             "kernels": kernels,
             "kv_gbs": world * total["kv_bytes"] / (ms_per_step * 1e-3) / 1e9,
+            "step_roofline": step_bound(total, ms_per_step, peaks, tensor_peak),
             "plan": steps[-1].info,
         }
         # Close the paper's control loop on the measured delay (Sec. 3.2-3.3, 3.5): one observation of (batched token
@@ -500,6 +621,22 @@ def main():
             rate, cores, sample, _, _ = time_oracle(sc, args.cpu_budget)
             line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                     "sample": sample}
+        if args.all_configs and world == 1:
+            # the other named workloads, briefly, so that all five are in this run's record (parity cases, not the
+            # headline: the line's value and roofline stay those of config.workload)
+            for ds in steps:
+                ds.close()
+            del steps, cache, flush_buf, host
+            torch.cuda.empty_cache()
+            line["all_configs"] = {}
+            for name in W.WORKLOADS:
+                if name == sc.name:
+                    continue
+                try:
+                    line["all_configs"][name] = quick_config(name, device, stream, peaks, peak_kind,
+                                                             with_oracle=not args.no_cpu_baseline)
+                except Exception as exc:
+                    line["all_configs"][name] = {"error": str(exc)}
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

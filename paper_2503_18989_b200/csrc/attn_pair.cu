@@ -144,10 +144,10 @@ struct Unit {
     int n;                                                        // key tiles of the range (at least 1)
 };
 __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* __restrict__ items, int unit) {
-    const int H = a.plan.num_heads;
-    const WorkItem it = items[unit / H];
+    const uint32_t e = __ldg(a.plan.tile_units + unit);      // item | head << 16
+    const WorkItem it = items[e & 0xffffu];
     Unit u;
-    u.h = unit % H;
+    u.h = (int)(e >> 16);
     u.hk = u.h / a.plan.group;
     u.r = it.req;
     u.P = a.plan.prefix_len[u.r];
@@ -429,7 +429,7 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
                     const int unit = bars->unit_slot[slot];
                     mbar_arrive(&bars->unit_empty[slot]);
                     if (unit < 0) break;
-                    const WorkItem it = items[unit / H];
+                    const WorkItem it = items[__ldg(a.plan.tile_units + unit) & 0xffffu];
                     const int n = max(1, (it.kv_end - it.kv_begin + kKeys - 1) / kKeys);
                     const int qs = un & 1;
                     const uint64_t qd = q_desc0 + (uint64_t)(qs * (kTileBytes >> 4));
@@ -488,7 +488,7 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
                     const int unit = bars->unit_slot[slot];
                     mbar_arrive(&bars->unit_empty[slot]);
                     if (unit < 0) break;
-                    const WorkItem it = items[unit / H];
+                    const WorkItem it = items[__ldg(a.plan.tile_units + unit) & 0xffffu];
                     const int n = max(1, (it.kv_end - it.kv_begin + kKeys - 1) / kKeys);
                     // the accumulators still hold the previous unit until its rows are in registers
                     if (un > 0) ok = mbar_wait(&bars->o_free, (un - 1) & 1, cx);
@@ -768,48 +768,36 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
     }
-}
-
-bool encode_q_map(CUtensorMap* map, bool bf16, const void* q, int T, int H) {
-    EncodeTiledFn fn = tma_encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)T};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)H * kD * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kRows};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(q), dims,
-              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    // The last CTA to get here (none draws units any more) leaves the unit counter at zero for the next call, which
+    // then needs no memset in front of it.  work_counter[1] counts the CTAs that have finished.
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(work_counter + 1, 1) == (int)gridDim.x - 1) {
+            work_counter[0] = 0;
+            work_counter[1] = 0;
+            __threadfence();
+        }
+    }
 }
 
 }  // namespace
 
 cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
-    CUtensorMap mq, mk, mv;
-    if (!encode_q_map(&mq, bf16, args.q, plan->total_rows, plan->num_heads) ||
-        !tma_encode_pool_map(&mk, bf16, args.cache.k_pool, kD, plan->num_pages, plan->num_kv_heads, args.cache.stride_page,
-                             args.cache.stride_token, args.cache.stride_head) ||
-        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, kD, plan->num_pages, plan->num_kv_heads, args.cache.stride_page,
-                             args.cache.stride_token, args.cache.stride_head))
-        return cudaErrorInvalidValue;
-    const int total_units = (int)plan->prefill_items.size() * plan->num_heads;
+    const CUtensorMap *mk = nullptr, *mv = nullptr;
+    const CUtensorMap* mq = plan_q_map(plan, args.q);
+    if (!mq || !plan_pool_maps(plan, args.cache, &mk, &mv)) return cudaErrorInvalidValue;
+    // the unit counter is zero at this point: the previous call's last CTA cleared it
+    const int total_units = (int)plan->tile_units.size();
     int32_t* counter = plan->dev.status + 1;
-    cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(int32_t), stream);
-    if (e != cudaSuccess) return e;
     // one cluster of two CTAs per pair of SMs, never more clusters than units
     int pairs = std::min(total_units, plan->num_sms / 2);
     if (const char* g = std::getenv("HAT_PAIR_GRID")) pairs = std::max(1, std::min(pairs, std::atoi(g)));
     const dim3 grid((unsigned)(2 * pairs));
-    if (bf16) {
-        e = cudaFuncSetAttribute(attn_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attn_pair_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, mq, mk, mv);
-    } else {
-        e = cudaFuncSetAttribute(attn_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attn_pair_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, mq, mk, mv);
-    }
+    auto kern = bf16 ? attn_pair_kernel<true> : attn_pair_kernel<false>;
+    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), kSmemBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, *mq, *mk, *mv);
     count_launch();
     return cudaGetLastError();
 }

@@ -381,7 +381,7 @@ cudaError_t launch_one(const hat_plan* plan, const AttnArgs& args, const CUtenso
                        cudaStream_t stream) {
     constexpr int smem = 1024 + 16 * D * 2 + kWarps * kSlots * 2 * (16 * D * 2) + kWarps * kSlots * 8 + 64;
     auto kern = attn_stream_kernel<BF16, D>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), smem);
     if (e != cudaSuccess) return e;
     kern<<<dim3(plan->num_kv_heads * plan->verify_subtiles, (unsigned)plan->verify_items.size()), kWarps * 32, smem, stream>>>(
         args, plan->dev.verify_items, plan->verify_subtiles, mk, mv);
@@ -401,15 +401,11 @@ bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int6
 
 cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
-    CUtensorMap mk, mv;
-    if (!tma_encode_pool_map(&mk, bf16, args.cache.k_pool, plan->head_dim, plan->num_pages, plan->num_kv_heads,
-                             args.cache.stride_page, args.cache.stride_token, args.cache.stride_head) ||
-        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, plan->head_dim, plan->num_pages, plan->num_kv_heads,
-                             args.cache.stride_page, args.cache.stride_token, args.cache.stride_head))
-        return cudaErrorInvalidValue;
+    const CUtensorMap *mk = nullptr, *mv = nullptr;
+    if (!plan_pool_maps(plan, args.cache, &mk, &mv)) return cudaErrorInvalidValue;
     if (plan->head_dim == 128)
-        return bf16 ? launch_one<true, 128>(plan, args, mk, mv, stream) : launch_one<false, 128>(plan, args, mk, mv, stream);
-    return bf16 ? launch_one<true, 64>(plan, args, mk, mv, stream) : launch_one<false, 64>(plan, args, mk, mv, stream);
+        return bf16 ? launch_one<true, 128>(plan, args, *mk, *mv, stream) : launch_one<false, 128>(plan, args, *mk, *mv, stream);
+    return bf16 ? launch_one<true, 64>(plan, args, *mk, *mv, stream) : launch_one<false, 64>(plan, args, *mk, *mv, stream);
 }
 
 }  // namespace hat

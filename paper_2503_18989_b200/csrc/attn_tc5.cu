@@ -95,10 +95,10 @@ struct Unit {
     __device__ __forceinline__ int tile_of(int t, int s) const { return split ? 2 * s + t : s; }
 };
 __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* __restrict__ items, int unit) {
-    const int H = a.plan.num_heads;
-    const WorkItem it = items[unit / H];
+    const uint32_t e = __ldg(a.plan.tile_units + unit);      // item | head << 16
+    const WorkItem it = items[e & 0xffffu];
     Unit u;
-    u.h = unit % H;
+    u.h = (int)(e >> 16);
     u.hk = u.h / a.plan.group;
     u.r = it.req;
     u.P = a.plan.prefix_len[u.r];
@@ -564,21 +564,19 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
     }
+    // The last CTA to get here (none draws units any more) leaves the unit counter at zero for the next call, which
+    // then needs no memset in front of it.  work_counter[1] counts the CTAs that have finished.
+    if (a.tail_reset && threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(work_counter + 1, 1) == (int)gridDim.x - 1) {
+            work_counter[0] = 0;
+            work_counter[1] = 0;
+            __threadfence();
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------- host side
-bool encode_q_map(CUtensorMap* map, bool bf16, const void* q, int T, int H) {
-    EncodeTiledFn fn = tma_encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)T};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)H * kD * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kRows};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(q), dims,
-              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
@@ -593,31 +591,22 @@ bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit,
                             bool reset_counter) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
-    CUtensorMap mq, mk, mv;
-    if (!encode_q_map(&mq, bf16, args.q, plan->total_rows, plan->num_heads) ||
-        !tma_encode_pool_map(&mk, bf16, args.cache.k_pool, kD, plan->num_pages, plan->num_kv_heads, args.cache.stride_page,
-                             args.cache.stride_token, args.cache.stride_head) ||
-        !tma_encode_pool_map(&mv, bf16, args.cache.v_pool, kD, plan->num_pages, plan->num_kv_heads, args.cache.stride_page,
-                             args.cache.stride_token, args.cache.stride_head))
-        return cudaErrorInvalidValue;
-    // one CTA per SM draws (item, head) units from a counter that is cleared on the stream first
-    const int total_units = (int)plan->prefill_items.size() * plan->num_heads;
+    const CUtensorMap *mk = nullptr, *mv = nullptr;
+    const CUtensorMap* mq = plan_q_map(plan, args.q);
+    if (!mq || !plan_pool_maps(plan, args.cache, &mk, &mv)) return cudaErrorInvalidValue;
+    // one CTA per SM draws units from a counter that is zero at this point: the previous call's last CTA cleared it
+    // (reset_counter); a grid that joins another one on the same counter leaves it alone
+    const int total_units = (int)plan->tile_units.size();
     int32_t* counter = plan->dev.status + 1;
-    cudaError_t e = cudaSuccess;
-    if (reset_counter) e = cudaMemsetAsync(counter, 0, sizeof(int32_t), stream);
-    if (e != cudaSuccess) return e;
+    AttnArgs a2 = args;
+    a2.tail_reset = reset_counter ? 1 : 0;
     int ctas = std::min(total_units, plan->num_sms);
     if (grid_limit > 0) ctas = std::min(ctas, grid_limit);
     const dim3 grid((unsigned)ctas);
-    if (bf16) {
-        e = cudaFuncSetAttribute(attn_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attn_tc5_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, mq, mk, mv);
-    } else {
-        e = cudaFuncSetAttribute(attn_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attn_tc5_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(args, plan->dev.prefill_items, total_units, counter, mq, mk, mv);
-    }
+    auto kern = bf16 ? attn_tc5_kernel<true> : attn_tc5_kernel<false>;
+    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), kSmemBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(a2, plan->dev.prefill_items, total_units, counter, *mq, *mk, *mv);
     count_launch();
     return cudaGetLastError();
 }

@@ -5,10 +5,13 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <vector>
 #include <queue>
 
 #include "hat_internal.h"
+#include "tma_desc.h"
 
 namespace hat {
 
@@ -17,6 +20,51 @@ static std::atomic<int64_t> g_launches{0};
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+cudaError_t smem_attr_once(const void* kernel, int bytes) {
+    struct Done { const void* kernel; int device; };
+    static std::mutex mu;
+    static std::vector<Done> done;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Done& d : done)
+        if (d.kernel == kernel && d.device == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done.push_back(Done{kernel, dev});
+    return e;
+}
+
+bool plan_pool_maps(const hat_plan* plan, const CacheView& c, const CUtensorMap** mk, const CUtensorMap** mv) {
+    MapCache& m = const_cast<hat_plan*>(plan)->maps;
+    if (!m.have_kv || m.k != c.k_pool || m.v != c.v_pool || m.stride_page != c.stride_page ||
+        m.stride_token != c.stride_token || m.stride_head != c.stride_head) {
+        const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
+        m.have_kv = false;
+        if (!tma_encode_pool_map(&m.mk, bf16, c.k_pool, plan->head_dim, plan->num_pages, plan->num_kv_heads, c.stride_page,
+                                 c.stride_token, c.stride_head) ||
+            !tma_encode_pool_map(&m.mv, bf16, c.v_pool, plan->head_dim, plan->num_pages, plan->num_kv_heads, c.stride_page,
+                                 c.stride_token, c.stride_head))
+            return false;
+        m.k = c.k_pool; m.v = c.v_pool;
+        m.stride_page = c.stride_page; m.stride_token = c.stride_token; m.stride_head = c.stride_head;
+        m.have_kv = true;
+    }
+    *mk = &m.mk; *mv = &m.mv;
+    return true;
+}
+
+const CUtensorMap* plan_q_map(const hat_plan* plan, const void* q) {
+    MapCache& m = const_cast<hat_plan*>(plan)->maps;
+    if (!m.have_q || m.q != q) {
+        m.have_q = false;
+        if (!tma_encode_q_map(&m.mq, plan->dtype == HAT_DTYPE_BF16, q, plan->total_rows, plan->num_heads)) return nullptr;
+        m.q = q;
+        m.have_q = true;
+    }
+    return &m.mq;
+}
 
 static int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
@@ -233,6 +281,23 @@ static void schedule(hat_plan* p, int num_sms, int tile_kernel) {
     std::stable_sort(p->verify_items.begin(), p->verify_items.end(), longer);
     std::stable_sort(p->prefill_items.begin(), p->prefill_items.end(), longer);
 
+    // Units of the persistent tcgen05 kernels, in the order the CTAs draw them: requests by their longest item first;
+    // inside a request head by head, and for each head all items of the request one after the other, so that the row
+    // blocks of one chunk (which read the same K/V of that head) run at the same time on neighbouring CTAs and meet in L2.
+    p->tile_units.clear();
+    if (use_tc5) {
+        std::vector<int> first_of_req(R, -1);
+        std::vector<std::vector<int>> group;
+        for (int i = 0; i < (int)p->prefill_items.size(); ++i) {
+            const int r = p->prefill_items[i].req;
+            if (first_of_req[r] < 0) { first_of_req[r] = (int)group.size(); group.emplace_back(); }
+            group[first_of_req[r]].push_back(i);
+        }
+        for (const std::vector<int>& g : group)          // items are sorted longest first, so groups are too
+            for (int h = 0; h < H; ++h)
+                for (int i : g) p->tile_units.push_back((uint32_t)i | ((uint32_t)h << 16));
+    }
+
     info.num_verify_items = (int32_t)p->verify_items.size();
     info.num_prefill_items = (int32_t)p->prefill_items.size();
     info.num_merge_rows = (int32_t)p->merge_rows.size();
@@ -260,6 +325,7 @@ static int upload(hat_plan* p) {
     size_t o_vi = blob_append(blob, p->verify_items);
     size_t o_pi = blob_append(blob, p->prefill_items);
     size_t o_mr = blob_append(blob, p->merge_rows);
+    size_t o_tu = blob_append(blob, p->tile_units);
     size_t o_tm = blob_append(blob, p->tree_mask);
     std::vector<int32_t> status(4, 0);
     size_t o_st = blob_append(blob, status);
@@ -280,6 +346,7 @@ static int upload(hat_plan* p) {
     d.verify_items = reinterpret_cast<const WorkItem*>(base + o_vi);
     d.prefill_items = reinterpret_cast<const WorkItem*>(base + o_pi);
     d.merge_rows = reinterpret_cast<const MergeRow*>(base + o_mr);
+    d.tile_units = reinterpret_cast<const uint32_t*>(base + o_tu);
     d.status = reinterpret_cast<int32_t*>(base + o_st);
     d.max_pages = p->max_pages;
     d.tree_mask = p->tree_mask.empty() ? nullptr : reinterpret_cast<const uint32_t*>(base + o_tm);
@@ -607,6 +674,7 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
     a.scale_log2 = sm_scale * 1.4426950408889634f;
     a.wait_cycles = plan->wait_cycles;
     a.withhold = plan->withhold_next;
+    a.tail_reset = 0;
     const_cast<hat_plan*>(plan)->withhold_next = 0;
 
     // Decode-phase (draft verification) requests first: their rows are final, and announced through the plan's event,
@@ -778,7 +846,7 @@ int hat_last_device_status(const hat_plan* plan, void* stream, int* out) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int32_t word = 0;
     cudaError_t e = cudaMemcpyAsync(&word, plan->dev.status, sizeof word, cudaMemcpyDeviceToHost, s);
-    if (e == cudaSuccess) e = cudaMemsetAsync(plan->dev.status, 0, sizeof word, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(plan->dev.status, 0, 4 * sizeof word, s);     // status, unit counter, finished CTAs
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
     *out = word == 0 ? HAT_OK : HAT_ERR_DEVICE_TIMEOUT;

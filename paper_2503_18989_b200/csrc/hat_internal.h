@@ -40,6 +40,7 @@ struct DevicePlan {
     const int32_t*  row_req;        // [T] request of each packed row
     const WorkItem* verify_items;
     const WorkItem* prefill_items;
+    const uint32_t* tile_units;     // tcgen05 tile kernels: unit -> prefill item (low 16 bits) | query head (high 16 bits), in draw order
     const MergeRow* merge_rows;
     const uint32_t* tree_mask;      // [T] or null: visible chunk positions of each row of a streaming-class request
     int32_t*        status;         // device status word (0 = ok)
@@ -69,6 +70,7 @@ struct AttnArgs {
     float       scale_log2;   // sm_scale * log2(e)
     long long   wait_cycles;  // bound of every device-side wait, in SM clock cycles
     int         withhold;     // self test: the tile kernel's producer skips its first V tile so that a wait runs out
+    int         tail_reset;   // the last CTA of the persistent tile kernel to finish clears the unit counter for the next call
 };
 
 // Key range of one split of the allocation-free streaming entry point, from lengths that nobody validated (they are
@@ -115,6 +117,21 @@ struct Timing {
 };
 }  // namespace hat
 
+#include <cuda.h>
+namespace hat {
+// Tensor maps of the last call, kept with what they were encoded for: a plan is reused for every layer of a step (and
+// by benchmarks for many steps) with the same pools and often the same q buffer, and encoding three maps per call is
+// a large part of the host time of a launch-bound step.
+struct MapCache {
+    const void* q = nullptr; const void* k = nullptr; const void* v = nullptr;
+    int64_t stride_page = 0, stride_token = 0, stride_head = 0;
+    bool have_q = false, have_kv = false;
+    CUtensorMap mq, mk, mv;
+};
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device instead of once per launch
+cudaError_t smem_attr_once(const void* kernel, int bytes);
+}  // namespace hat
+
 struct hat_plan {
     // geometry the plan was made for
     int32_t dtype, num_pages, num_heads, num_kv_heads, head_dim, max_pages, num_requests, total_rows;   // num_heads: query heads
@@ -125,6 +142,7 @@ struct hat_plan {
     int num_sms;
     std::vector<int32_t> cu_chunk, prefix_len, chunk_len, block_table, row_req;
     std::vector<hat::WorkItem> verify_items, prefill_items;
+    std::vector<uint32_t> tile_units;   // (item, head) of every unit of the tcgen05 tile kernels, in the order they are drawn
     std::vector<hat::MergeRow> merge_rows;
     int64_t part_rows;          // partial rows in the workspace
     hat_plan_info info;
@@ -142,6 +160,7 @@ struct hat_plan {
     cudaEvent_t ev_fork, ev_join;
     long long wait_cycles;      // bound of device-side waits (default: about a second)
     int withhold_next;          // self test of the bounded waits: applies to the next attention call only
+    hat::MapCache maps;         // see MapCache (updated through const_cast by the launchers: one call at a time per plan)
     void* dev_blob;             // one allocation holding every device array
     hat::DevicePlan dev;
 };
@@ -170,4 +189,11 @@ bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int6
 cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
 void count_launch(int n = 1);
 void set_last_cuda_error(int e);   // what hat_last_cuda_error() returns on this thread
+}  // namespace hat
+
+namespace hat {
+// The plan's cached tensor maps for these pools / this q buffer, encoded again only when a pointer or a stride changed.
+// Return null when no map can be built.  (Defined in hat_api.cu.)
+bool plan_pool_maps(const hat_plan* plan, const CacheView& cache, const CUtensorMap** mk, const CUtensorMap** mv);
+const CUtensorMap* plan_q_map(const hat_plan* plan, const void* q);
 }  // namespace hat
