@@ -45,6 +45,7 @@ extern "C" {
 #define HAT_ERR_CUDA                 -5  /* a CUDA runtime call failed; see hat_last_cuda_error */
 #define HAT_ERR_DEVICE_TIMEOUT       -6  /* a bounded device-side wait gave up (reported by hat_last_device_status) */
 #define HAT_ERR_TOO_LARGE            -7  /* a size exceeds a documented fixed maximum */
+#define HAT_ERR_DEVICE_BOUNDS         -8  /* debug build only: a device-side index check failed (reported by hat_last_device_status) */
 
 #define HAT_DTYPE_FP16 0
 #define HAT_DTYPE_BF16 1
@@ -291,7 +292,9 @@ int hat_plan_wait_verify(const hat_plan* plan);
 
 /*
  * Read and clear the device-side status word of a plan (synchronises
- * `stream`).  *out is HAT_OK, or HAT_ERR_DEVICE_TIMEOUT if a bounded wait
+ * `stream`).  *out is HAT_OK, HAT_ERR_DEVICE_BOUNDS (only a library built with
+ * -DHAT_DEBUG_BOUNDS checks: a block-table column, page id, ring slot, TMEM column or output row was out of range;
+ * the access was skipped or clamped, nothing trapped), or HAT_ERR_DEVICE_TIMEOUT if a bounded wait
  * inside a kernel gave up since the word was last read; the results of the
  * calls in between are then undefined, but the kernels have exited normally
  * and the context stays usable.

@@ -14,7 +14,8 @@ from typing import Optional
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libhat.so")
+# HAT_LIB=debug loads the build with device-side index checks (python -m paper_2503_18989_b200.build --debug)
+LIB_PATH = os.path.join(_HERE, "libhat_debug.so" if os.environ.get("HAT_LIB") == "debug" else "libhat.so")
 
 HAT_OK = 0
 HAT_ERR_INVALID_ARG = -1
@@ -24,6 +25,7 @@ HAT_ERR_WORKSPACE_TOO_SMALL = -4
 HAT_ERR_CUDA = -5
 HAT_ERR_DEVICE_TIMEOUT = -6
 HAT_ERR_TOO_LARGE = -7
+HAT_ERR_DEVICE_BOUNDS = -8
 HAT_DTYPE_FP16 = 0
 HAT_DTYPE_BF16 = 1
 HAT_PLAN_HOST_ONLY = 1

@@ -39,17 +39,29 @@ def is_stale() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library; returns its path."""
+LIB_DEBUG = os.path.join(HERE, "libhat_debug.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile every .cu under csrc/ into one shared library; returns its path.
+    debug=True builds libhat_debug.so with -DHAT_DEBUG_BOUNDS: device-side range checks of block-table lookups, page
+    ids, ring slots, TMEM columns and output rows that report through the plan's status word instead of trapping
+    (load it with HAT_LIB=debug)."""
+    if debug:
+        return _build(LIB_DEBUG, "_build_debug", ["-DHAT_DEBUG_BOUNDS"], verbose)
     if not force and not is_stale():
         return LIB
+    return _build(LIB, "_build", [], verbose)
+
+
+def _build(lib: str, obj_name: str, extra, verbose: bool) -> str:
     objs = []
-    obj_dir = os.path.join(HERE, "_build")
+    obj_dir = os.path.join(HERE, obj_name)
     os.makedirs(obj_dir, exist_ok=True)
     procs = []
     for src in sources():
         obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", src, "-o", obj]
+        cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
@@ -65,11 +77,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
             print(f"nvcc failed on {src}", file=sys.stderr)
     if failed:
         raise RuntimeError("CUDA build failed")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart_static", "-ldl", "-lpthread", "-lrt"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

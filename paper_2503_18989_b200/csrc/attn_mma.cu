@@ -139,7 +139,7 @@ attn_mma_kernel(AttnArgs a, const WorkItem* __restrict__ items) {
             const int key = kb + row;
             const uint32_t off = swz<D>(row, c);
             if (key < item.kv_end) {
-                const int page = __ldg(table + key / kPageSize);
+                const int page = HAT_IN_RANGE(__ldg(table + HAT_IN_RANGE(key / kPageSize, a.plan.max_pages, a.plan.status)), a.plan.num_pages, a.plan.status);
                 const int64_t e = (int64_t)page * a.cache.stride_page + (int64_t)(key % kPageSize) * a.cache.stride_token +
                                   head_off + c * 8;
                 cp_async16(kdst + off, kpool + e);

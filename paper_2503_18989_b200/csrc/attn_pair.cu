@@ -131,7 +131,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
         if (clock64() - t0 > cx.bars->wait_cycles) {
             cx.bars->abort_flag = 1;
             st_cluster_b32(cx.peer_abort, 1u);
-            atomicExch(cx.status, 1);
+            atomicOr(cx.status, 1);
             return false;
         }
     }
@@ -290,13 +290,15 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
             // The page id of the NEXT tile is fetched while this tile's boxes are issued.
             const int total_pages = (u.kv_end - u.kv_begin + kPageSize - 1) / kPageSize;
             const int kpg = 4 * (int)rank + (lane >> 1), khalf = lane & 1;
-            int page = (lane < 8 && kpg < total_pages) ? __ldg(table + kpg) : 0;
+            HAT_CHECK(u.kv_begin / kPageSize + total_pages <= a.plan.max_pages, cx.status);
+            int page = (lane < 8 && kpg < total_pages) ? HAT_IN_RANGE(__ldg(table + kpg), a.plan.num_pages, cx.status) : 0;
             for (int j = 0; j < u.n; ++j, ++g) {
                 const int sk = g % kStagesK;
                 const int npages = min(8, total_pages - 8 * j);                                   // pages of this tile: 1..8
                 const int nk = max(0, min(4, npages - 4 * (int)rank));                            // K pages this CTA loads
                 const int next_pg = 8 * (j + 1) + kpg;
-                const int page_next = (lane < 8 && next_pg < total_pages) ? __ldg(table + next_pg) : 0;
+                const int page_next = (lane < 8 && next_pg < total_pages) ? HAT_IN_RANGE(__ldg(table + next_pg), a.plan.num_pages, cx.status) : 0;
+                HAT_CHECK(sk < kStagesK, cx.status);
                 PH_ADD(2, tq0);
                 if (g >= kStagesK) ok = mbar_wait(&bars->k_empty[sk], ((g / kStagesK) & 1) ^ 1, cx);
                 ok = __all_sync(0xffffffffu, ok);
@@ -336,12 +338,14 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
             const Unit u = decode_unit(a, items, unit);
             const int32_t* __restrict__ table = a.plan.block_table + (int64_t)u.r * a.plan.max_pages + u.kv_begin / kPageSize;
             const int total_pages = (u.kv_end - u.kv_begin + kPageSize - 1) / kPageSize;
-            int page = (lane < 8 && lane < total_pages) ? __ldg(table + lane) : 0;
+            HAT_CHECK(u.kv_begin / kPageSize + total_pages <= a.plan.max_pages, cx.status);
+            int page = (lane < 8 && lane < total_pages) ? HAT_IN_RANGE(__ldg(table + lane), a.plan.num_pages, cx.status) : 0;
             for (int j = 0; j < u.n; ++j, ++g) {
                 const int sv = g % kStagesV;
                 const int npages = min(8, total_pages - 8 * j);
                 const int next_pg = 8 * (j + 1) + lane;
-                const int page_next = (lane < 8 && next_pg < total_pages) ? __ldg(table + next_pg) : 0;
+                const int page_next = (lane < 8 && next_pg < total_pages) ? HAT_IN_RANGE(__ldg(table + next_pg), a.plan.num_pages, cx.status) : 0;
+                HAT_CHECK(sv < kStagesV, cx.status);
                 if (g >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((g / kStagesV) & 1) ^ 1, cx);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -716,6 +720,7 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
                 float* obase; float* lbase; int64_t orow;
                 if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
                 else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
+                HAT_CHECK(orow >= 0 && orow < (u.part < 0 ? (int64_t)a.plan.total_rows : a.part_rows), cx.status);
                 if (u.part < 0 && a.out16 != nullptr) {
                     // final rows in the 16-bit output type: 128 bytes per row and warpgroup
                     uint16_t* dst16 = static_cast<uint16_t*>(a.out16) + (orow * H + u.h) * kD + w * 64;

@@ -134,7 +134,7 @@ attn_stream_kernel(AttnArgs a, const WorkItem* __restrict__ items, int n_sub, co
         __syncwarp();
         if (lane < 2 * HALVES) {
             const int is_v = lane / HALVES, half = lane % HALVES;
-            const int page = __ldg(table + kb / kPageSize);
+            const int page = HAT_IN_RANGE(__ldg(table + HAT_IN_RANGE(kb / kPageSize, a.plan.max_pages, a.plan.status)), a.plan.num_pages, a.plan.status);
             const uint32_t dst = ring + slot * SLOT_BYTES + is_v * PAGE_BYTES + half * 2048;
             const CUtensorMap* map = is_v ? &map_v : &map_k;
             asm volatile(

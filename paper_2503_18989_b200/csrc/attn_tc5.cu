@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barrie
         if (b->abort_flag) return false;
         if (clock64() - t0 > b->wait_cycles) {
             b->abort_flag = 1;
-            atomicExch(status, 1);
+            atomicOr(status, 1);
             return false;
         }
     }
@@ -198,7 +198,9 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                 const int kb = u.kv_begin + j * kKeys;
                 const int npages = (min(u.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
                 int page = 0;
-                if (lane < 16 && pg < npages) page = __ldg(table + kb / kPageSize + pg);
+                if (lane < 16 && pg < npages)
+                    page = HAT_IN_RANGE(__ldg(table + HAT_IN_RANGE(kb / kPageSize + pg, a.plan.max_pages, status)), a.plan.num_pages, status);
+                HAT_CHECK(sk < kStagesK && sv < kStagesV, status);
                 if (kt >= kStagesK) ok = mbar_wait(&bars->k_empty[sk], ((kt / kStagesK) & 1) ^ 1, bars, status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -298,6 +300,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         tc_fence_after();
                         const uint64_t vd = v_desc0 + (uint64_t)(st * (kTileBytes >> 4));
                         const uint32_t tp = tmem + qt * 128, to = tmem + 256 + qt * 128;
+                        HAT_CHECK((to & 0xffffu) + 128 <= 512 && (tp & 0xffffu) + 128 <= 256, status);
 #pragma unroll
                         for (int ks = 0; ks < kKeys / 16; ++ks) {
                             // 16 keys = 2048 bytes of every 64-column slab; slabs 16 KiB apart (leading), 8-key groups 1 KiB apart
@@ -520,6 +523,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         float* obase; float* lbase; int64_t orow;
                         if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
                         else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
+                        HAT_CHECK(orow >= 0 && orow < (u.part < 0 ? (int64_t)a.plan.total_rows : a.part_rows), status);
                         float* dst = obase + (orow * H + u.h) * kD;
                         if (u.part < 0 && a.out16 != nullptr) {
                             // final rows in the 16-bit output type: 256 bytes per row, eight 32-byte stores

@@ -354,6 +354,7 @@ static int upload(hat_plan* p) {
     d.num_kv_heads = p->num_kv_heads;
     d.group = p->num_heads / p->num_kv_heads;
     d.total_rows = p->total_rows;
+    d.num_pages = p->num_pages;
     return HAT_OK;
 }
 
@@ -390,6 +391,7 @@ const char* hat_status_string(int status) {
         case HAT_ERR_CUDA: return "CUDA error";
         case HAT_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
         case HAT_ERR_TOO_LARGE: return "size exceeds a fixed maximum";
+        case HAT_ERR_DEVICE_BOUNDS: return "device-side index check failed (debug build)";
         default: return "unknown status";
     }
 }
@@ -671,6 +673,7 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
     const int64_t H = plan->num_heads, d = plan->head_dim;
     const size_t part_out_bytes = ((size_t)plan->part_rows * H * d * 4 + 255) / 256 * 256;
     a.part_lse = need ? reinterpret_cast<float*>(static_cast<char*>(workspace) + part_out_bytes) : nullptr;
+    a.part_rows = plan->part_rows;
     a.scale_log2 = sm_scale * 1.4426950408889634f;
     a.wait_cycles = plan->wait_cycles;
     a.withhold = plan->withhold_next;
@@ -849,7 +852,7 @@ int hat_last_device_status(const hat_plan* plan, void* stream, int* out) {
     if (e == cudaSuccess) e = cudaMemsetAsync(plan->dev.status, 0, 4 * sizeof word, s);     // status, unit counter, finished CTAs
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
-    *out = word == 0 ? HAT_OK : HAT_ERR_DEVICE_TIMEOUT;
+    *out = word == 0 ? HAT_OK : (word & 1) ? HAT_ERR_DEVICE_TIMEOUT : HAT_ERR_DEVICE_BOUNDS;
     return HAT_OK;
 }
 

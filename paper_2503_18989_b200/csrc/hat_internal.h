@@ -49,6 +49,7 @@ struct DevicePlan {
     int32_t         num_kv_heads;   // K/V heads (pools, k_new, v_new)
     int32_t         group;          // query heads per K/V head
     int32_t         total_rows;
+    int32_t         num_pages;      // pages in the pools (index checks of the debug build)
 };
 
 struct CacheView {
@@ -67,6 +68,7 @@ struct AttnArgs {
     float*      lse;          // [T][H]
     float*      part_out;     // [part_rows][H][d]
     float*      part_lse;     // [part_rows][H]
+    int64_t     part_rows;    // partial rows the workspace holds (index checks of the debug build)
     float       scale_log2;   // sm_scale * log2(e)
     long long   wait_cycles;  // bound of every device-side wait, in SM clock cycles
     int         withhold;     // self test: the tile kernel's producer skips its first V tile so that a wait runs out
@@ -94,6 +96,22 @@ inline StaticRange static_key_range(int prefix_len, int chunk_len, int max_rows,
     if (e > N) e = N;
     return StaticRange{(int)P, (int)C, (int)b, (int)e};
 }
+
+// Debug build (-DHAT_DEBUG_BOUNDS): indices that the release build trusts (they were validated on the host, or follow
+// from the kernel's own arithmetic) are range-checked on the device; a violation raises bit 1 of the plan's status
+// word (hat_last_device_status then reports HAT_ERR_DEVICE_BOUNDS) and never traps.  HAT_IN_RANGE returns the index
+// clamped into [0, n) so that the access that follows stays inside the array either way.
+#if defined(__CUDACC__) && defined(HAT_DEBUG_BOUNDS)
+__device__ __forceinline__ int hat_in_range(int i, int n, int32_t* status) {
+    if (i < 0 || i >= n) { atomicOr(status, 2); return i < 0 ? 0 : (n > 0 ? n - 1 : 0); }
+    return i;
+}
+#define HAT_IN_RANGE(i, n, status) hat_in_range((i), (n), (status))
+#define HAT_CHECK(cond, status) do { if (!(cond)) atomicOr((status), 2); } while (0)
+#else
+#define HAT_IN_RANGE(i, n, status) (i)
+#define HAT_CHECK(cond, status) do { } while (0)
+#endif
 
 #ifdef __CUDACC__
 // Two fp32 values rounded to nearest into one 32-bit word of the 16-bit output type (low half = first value).

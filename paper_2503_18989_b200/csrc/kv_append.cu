@@ -32,9 +32,10 @@ kv_append_kernel(DevicePlan plan, int64_t stride_page, int64_t stride_token, int
         const int within = (int)(idx - (int64_t)t * vec_per_row);
         const int h = within / vec_per_head;
         const int c = within - h * vec_per_head;
-        const int r = plan.row_req[t];
+        const int r = plan.row_req[HAT_IN_RANGE(t, plan.total_rows, plan.status)];
         const int pos = plan.prefix_len[r] + (t - plan.cu_chunk[r]);     // logical token index
-        const int page = plan.block_table[(int64_t)r * plan.max_pages + pos / kPageSize];
+        const int page = HAT_IN_RANGE(plan.block_table[(int64_t)r * plan.max_pages + HAT_IN_RANGE(pos / kPageSize, plan.max_pages, plan.status)],
+                                      plan.num_pages, plan.status);
         const int slot = pos % kPageSize;
         // strides are multiples of 8 elements, so the offset in 16-byte vectors is exact
         const int64_t dst = ((int64_t)page * stride_page + (int64_t)slot * stride_token + (int64_t)h * stride_head) / 8 + c;

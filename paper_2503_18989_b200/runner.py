@@ -17,6 +17,32 @@ def _dev_u16(a: np.ndarray, device) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(device, non_blocking=False)
 
 
+_GUARD_BYTES = 1024      # canary zone in front of and behind every buffer the library writes
+_GUARD_BYTE = 0x5A
+
+
+class _Guarded:
+    """A device buffer between two canary zones: `view` is what the library gets, intact() tells whether anything
+    was written outside it."""
+
+    def __init__(self, shape, dtype, fill, device):
+        n = 1
+        for x in shape:
+            n *= int(x)
+        item = torch.empty(0, dtype=dtype).element_size()
+        self.nbytes = n * item
+        pad = (-self.nbytes) % 256                       # keep the rear zone (and the next allocation) aligned
+        self.raw = torch.full((_GUARD_BYTES + self.nbytes + pad + _GUARD_BYTES,), _GUARD_BYTE, dtype=torch.uint8, device=device)
+        self.view = self.raw[_GUARD_BYTES:_GUARD_BYTES + self.nbytes].view(dtype).view(*shape)
+        if fill is not None:
+            self.view.fill_(fill)
+
+    def intact(self) -> bool:
+        front = self.raw[:_GUARD_BYTES]
+        rear = self.raw[_GUARD_BYTES + self.nbytes:]
+        return bool((front == _GUARD_BYTE).all().item()) and bool((rear == _GUARD_BYTE).all().item())
+
+
 class DeviceCache:
     """K and V pools of one layer on the device."""
 
@@ -49,10 +75,14 @@ class DeviceStep:
         self.q = _dev_u16(step.q, dev)
         self.k_new = _dev_u16(step.k_new, dev)
         self.v_new = _dev_u16(step.v_new, dev)
-        self.out = torch.full((T, H, d), float("nan"), dtype=torch.float32, device=dev)
-        self.lse = torch.full((T, H), float("nan"), dtype=torch.float32, device=dev)
+        # every buffer the library writes sits between canary zones (checked by canaries_intact)
+        self._g_out = _Guarded((T, H, d), torch.float32, float("nan"), dev)
+        self._g_lse = _Guarded((T, H), torch.float32, float("nan"), dev)
+        self.out, self.lse = self._g_out.view, self._g_lse.view
         self.workspace_bytes = B.hat_plan_workspace_bytes(self.plan)
-        self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=dev)
+        self._g_ws = _Guarded((max(self.workspace_bytes, 256),), torch.uint8, None, dev)
+        self.workspace = self._g_ws.view
+        self._g_out16 = None
 
     def append(self, stream: int = 0) -> None:
         B.hat_kv_append(self.cache.desc, self.plan, self.k_new, self.v_new, stream)
@@ -60,7 +90,8 @@ class DeviceStep:
     def attend16(self, fused_append: bool = True, sm_scale: float = 0.0, stream: int = 0) -> None:
         """The same step with the output in the cache's 16-bit type (self.out16, allocated on first use)."""
         if getattr(self, "out16", None) is None:
-            self.out16 = torch.full(self.out.shape, -1, dtype=torch.int16, device=self.out.device)
+            self._g_out16 = _Guarded(tuple(self.out.shape), torch.int16, -1, self.out.device)
+            self.out16 = self._g_out16.view
         B.hat_chunk_attention_out16(self.cache.desc, self.plan, self.q,
                                     self.k_new if fused_append else None, self.v_new if fused_append else None,
                                     self.out16, self.lse, sm_scale, self.workspace, self.workspace_bytes, stream)
@@ -73,6 +104,11 @@ class DeviceStep:
     def results(self):
         torch.cuda.synchronize(self.cache.device)
         return self.out.cpu().numpy(), self.lse.cpu().numpy()
+
+    def canaries_intact(self) -> bool:
+        """No byte outside out / lse / workspace (/ out16) was written."""
+        torch.cuda.synchronize(self.cache.device)
+        return all(g.intact() for g in (self._g_out, self._g_lse, self._g_ws, self._g_out16) if g is not None)
 
     def close(self):
         self.plan.close()
@@ -88,7 +124,10 @@ def run_scenario(sc: Scenario, device="cuda:0", fused_append: bool = True):
             ds.append()
         ds.attend(fused_append=fused_append)
         res.append(ds.results())
-        if B.hat_last_device_status(ds.plan) != B.HAT_OK:
-            raise RuntimeError("device-side wait timed out")
+        status = B.hat_last_device_status(ds.plan)
+        if status != B.HAT_OK:
+            raise RuntimeError(f"device status {status}: {B.hat_status_string(status)}")
+        if not ds.canaries_intact():
+            raise RuntimeError("a canary zone around out / lse / workspace was overwritten")
         ds.close()
     return cache, res

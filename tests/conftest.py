@@ -17,7 +17,8 @@ def hat_lib():
     """Build (if stale) and load the CUDA library; a build failure fails the test."""
     from paper_2503_18989_b200 import build as hat_build
     from paper_2503_18989_b200 import binding
-    hat_build.build()
+    # HAT_LIB=debug runs the suite against the build with device-side index checks
+    hat_build.build(debug=os.environ.get("HAT_LIB") == "debug")
     return binding.lib()
 
 
