@@ -38,10 +38,11 @@ using namespace tc5;
 
 constexpr int kRows = 128;      // query rows per CTA (MMA M)
 constexpr int kKeys = 128;      // keys per tile (MMA N of S, K extent of PV)
-constexpr int kD = 128;         // head_dim
 constexpr int kStagesK = 2;     // ring slots for K tiles
 constexpr int kStagesV = 3;     // ring slots for V tiles (V is requested later in a step than K, so it gets the deeper ring)
-constexpr uint32_t kTileBytes = kKeys * kD * 2;          // 32 KiB: one K or V tile, or the Q tile
+// one K or V tile, or the Q tile: 128 rows of head_dim 16-bit values (32 KiB at head_dim 128, 16 KiB at 64), stored as
+// head_dim / 64 slabs of 64 columns
+template <int D> constexpr uint32_t tile_bytes() { return kKeys * D * 2; }
 constexpr uint32_t kSlabBytes = kKeys * 64 * 2;          // 16 KiB: 64 columns of 128 rows
 constexpr uint32_t kPageBoxBytes = 16 * 64 * 2;          // 2 KiB: one TMA box (16 tokens x 64 columns)
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
@@ -60,8 +61,8 @@ struct __align__(8) Barriers {
     volatile int unit_slot[2];                              // unit index, or -1 when the work has run out
     float2 xchg[kRows];                                     // split units: per row, chain 1's reference maximum and row sum
 };
-constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (2 + kStagesK + kStagesV) + sizeof(Barriers);
-static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
+template <int D> constexpr uint32_t smem_bytes() { return 1024 /*alignment slack*/ + tile_bytes<D>() * (2 + kStagesK + kStagesV) + sizeof(Barriers); }
+static_assert(smem_bytes<128>() <= 227 * 1024, "shared memory of one CTA");
 constexpr int kThreads = 320;   // producer warp, MMA warp, two softmax warpgroups
 
 // Bounded wait.  Returns false if the wait gave up or another role already did.
@@ -115,11 +116,13 @@ __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, const WorkItem* _
     return u;
 }
 
-template <bool BF16>
+template <bool BF16, int kD>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units, int32_t* work_counter,
                 const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v) {
+    constexpr uint32_t kTileBytes = tile_bytes<kD>();
+    constexpr int kHalves = kD / 64;                             // 64-column slabs (and TMA boxes per page) of a tile
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: the swizzle pattern and the matrix descriptors assume it
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -163,7 +166,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
     if (warp == 0) {
         // ------------------------------------------------------------------ unit fetch + TMA producer
         // lane l < 16 moves box (page l/2 of the tile, column half l%2)
-        const int pg = lane >> 1, half = lane & 1;
+        const int pg = lane / kHalves, half = lane % kHalves;
         int kt = 0;                                              // K/V tiles issued so far, over all units
         bool ok = true;
         for (int un = 0; ok; ++un) {
@@ -190,32 +193,32 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
             }
             if (lane == 0) mbar_expect_tx(&bars->q_full, u.nq * kTileBytes);
             __syncwarp();
-            if (lane < 2 * u.nq)      // lane = 2 * (query tile) + (column half)
-                tma_load_3d(smem_u32(q_tiles) + (lane >> 1) * kTileBytes + (lane & 1) * kSlabBytes, &map_q, (lane & 1) * 64, u.h,
-                            u.row_base + u.row0 + (lane >> 1) * kRows, &bars->q_full);
+            if (lane < kHalves * u.nq)      // lane = kHalves * (query tile) + (column half)
+                tma_load_3d(smem_u32(q_tiles) + (lane / kHalves) * kTileBytes + (lane % kHalves) * kSlabBytes, &map_q, (lane % kHalves) * 64, u.h,
+                            u.row_base + u.row0 + (lane / kHalves) * kRows, &bars->q_full);
             for (int j = 0; j < u.n_all; ++j, ++kt) {
                 const int sk = kt % kStagesK, sv = kt % kStagesV;
                 const int kb = u.kv_begin + j * kKeys;
                 const int npages = (min(u.kv_end, kb + kKeys) - kb + kPageSize - 1) / kPageSize;
                 int page = 0;
-                if (lane < 16 && pg < npages)
+                if (lane < 8 * kHalves && pg < npages)
                     page = HAT_IN_RANGE(__ldg(table + HAT_IN_RANGE(kb / kPageSize + pg, a.plan.max_pages, status)), a.plan.num_pages, status);
                 HAT_CHECK(sk < kStagesK && sv < kStagesV, status);
                 if (kt >= kStagesK) ok = mbar_wait(&bars->k_empty[sk], ((kt / kStagesK) & 1) ^ 1, bars, status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (lane == 0) mbar_expect_tx(&bars->k_full[sk], npages * 2 * kPageBoxBytes);
+                if (lane == 0) mbar_expect_tx(&bars->k_full[sk], npages * kHalves * kPageBoxBytes);
                 __syncwarp();
-                if (lane < 16 && pg < npages)
+                if (lane < 8 * kHalves && pg < npages)
                     tma_load_4d(smem_u32(k_ring) + sk * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_k, half * 64, 0,
                                 u.hk, page, &bars->k_full[sk]);
                 if (kt >= kStagesV) ok = mbar_wait(&bars->v_empty[sv], ((kt / kStagesV) & 1) ^ 1, bars, status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (a.withhold && kt == 0) continue;         // self test: this V tile never arrives, its consumers give up
-                if (lane == 0) mbar_expect_tx(&bars->v_full[sv], npages * 2 * kPageBoxBytes);
+                if (lane == 0) mbar_expect_tx(&bars->v_full[sv], npages * kHalves * kPageBoxBytes);
                 __syncwarp();
-                if (lane < 16 && pg < npages)
+                if (lane < 8 * kHalves && pg < npages)
                     tma_load_4d(smem_u32(v_ring) + sv * kTileBytes + half * kSlabBytes + pg * kPageBoxBytes, &map_v, half * 64, 0,
                                 u.hk, page, &bars->v_full[sv]);
             }
@@ -433,7 +436,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                     }
                     if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
+                        for (int c = 0; c < kD / 32; ++c) {
                             uint32_t o[32];
                             tmem_ld32(tm_o + c * 32, o);
                             tmem_ld_wait();
@@ -451,8 +454,9 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         if (!ok) break;
                         unsigned char* vt = v_ring + (kt % kStagesV) * kTileBytes;
                         const int first = u.kv_end - kb;
-                        for (int idx = wg_tid; idx < (kKeys - first) * 16; idx += 128) {
-                            const int row = first + idx / 16, part = idx % 16;     // 16 vectors of 16 bytes per 256-byte row
+                        constexpr int kVecs = kD / 8;                              // 16-byte vectors per row
+                        for (int idx = wg_tid; idx < (kKeys - first) * kVecs; idx += 128) {
+                            const int row = first + idx / kVecs, part = idx % kVecs;
                             *reinterpret_cast<uint4*>(vt + (part >> 3) * kSlabBytes + row * 128 + (part & 7) * 16) = make_uint4(0, 0, 0, 0);
                         }
                         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -483,7 +487,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                 } else {
                     if (n_mine > 0) {
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) tmem_ld32(tm_o + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
+                        for (int c = 0; c < kD / 32; ++c) tmem_ld32(tm_o + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
                         tmem_ld_wait();
                     } else {
 #pragma unroll
@@ -502,7 +506,7 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
                         l = l * w0 + other.y * w1;
                         m_used = m_new;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
+                        for (int c = 0; c < kD / 16; ++c) {
                             uint32_t o1[16];
                             tmem_ld16(tm_o + 128 + c * 16, o1);      // the second chain's accumulator: next 128 columns
                             tmem_ld_wait();
@@ -585,11 +589,11 @@ attn_tc5_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units,
 
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                           int64_t stride_head) {
-    if (head_dim != kD || num_pages <= 0) return false;
+    if ((head_dim != 64 && head_dim != 128) || num_pages <= 0) return false;
     CUtensorMap m;
     // the encoder checks alignment and ranges only; any 16-byte aligned address will do for the probe
-    return tma_encode_pool_map(&m, dtype == HAT_DTYPE_BF16, reinterpret_cast<const void*>(uintptr_t(1) << 30), kD, num_pages,
-                               H, stride_page, stride_token, stride_head);
+    return tma_encode_pool_map(&m, dtype == HAT_DTYPE_BF16, reinterpret_cast<const void*>(uintptr_t(1) << 30), head_dim,
+                               num_pages, H, stride_page, stride_token, stride_head);
 }
 
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit,
@@ -607,10 +611,13 @@ cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStre
     int ctas = std::min(total_units, plan->num_sms);
     if (grid_limit > 0) ctas = std::min(ctas, grid_limit);
     const dim3 grid((unsigned)ctas);
-    auto kern = bf16 ? attn_tc5_kernel<true> : attn_tc5_kernel<false>;
-    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), kSmemBytes);
+    const bool d128 = plan->head_dim == 128;
+    auto kern = d128 ? (bf16 ? attn_tc5_kernel<true, 128> : attn_tc5_kernel<false, 128>)
+                     : (bf16 ? attn_tc5_kernel<true, 64> : attn_tc5_kernel<false, 64>);
+    const uint32_t smem = d128 ? smem_bytes<128>() : smem_bytes<64>();
+    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, stream>>>(a2, plan->dev.prefill_items, total_units, counter, *mq, *mk, *mv);
+    kern<<<grid, kThreads, smem, stream>>>(a2, plan->dev.prefill_items, total_units, counter, *mq, *mk, *mv);
     count_launch();
     return cudaGetLastError();
 }

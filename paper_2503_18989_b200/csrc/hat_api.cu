@@ -59,7 +59,7 @@ const CUtensorMap* plan_q_map(const hat_plan* plan, const void* q) {
     MapCache& m = const_cast<hat_plan*>(plan)->maps;
     if (!m.have_q || m.q != q) {
         m.have_q = false;
-        if (!tma_encode_q_map(&m.mq, plan->dtype == HAT_DTYPE_BF16, q, plan->total_rows, plan->num_heads)) return nullptr;
+        if (!tma_encode_q_map(&m.mq, plan->dtype == HAT_DTYPE_BF16, q, plan->total_rows, plan->num_heads, plan->head_dim)) return nullptr;
         m.q = q;
         m.have_q = true;
     }
@@ -495,8 +495,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) { delete p; return cuda_fail(e); }
     }
-    // the tcgen05 tile kernel needs head_dim 128 and a pool layout a TMA descriptor can express
-    bool use_tc5 = p->head_dim == 128;
+    // the tcgen05 tile kernels need a pool layout a TMA descriptor can express (the CTA-pair one also head_dim 128)
+    bool use_tc5 = true;
     if (const char* k = std::getenv("HAT_PREFILL_KERNEL"))
         if (std::strcmp(k, "mma") == 0) use_tc5 = false;
     if (use_tc5 && !p->host_only)
@@ -505,7 +505,7 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->num_sms = num_sms;
     int tile_kernel = use_tc5 ? 1 : 0;
     if (const char* k = std::getenv("HAT_PREFILL_KERNEL"))
-        if (use_tc5 && std::strcmp(k, "pair") == 0) tile_kernel = 3;
+        if (use_tc5 && p->head_dim == 128 && std::strcmp(k, "pair") == 0) tile_kernel = 3;
     schedule(p, num_sms, tile_kernel);
     // the streaming kernel takes its pages by TMA when a descriptor can be built for the pool layout
     bool stream_tma = true;

@@ -193,7 +193,7 @@ cudaError_t launch_attn_mma(const hat_plan* plan, const AttnArgs& args, bool ver
 cudaError_t launch_rope(const hat_plan* plan, int heads, float theta, int interleaved, const void* src, void* dst,
                         const CacheView* cache, void* k_pool, void* v_pool, const void* v_new, cudaStream_t stream);
 cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, int first_row, int num_rows, cudaStream_t stream);
-// tcgen05 tile kernel (head_dim 128): whether a TMA descriptor can be built for this pool layout, and the launcher
+// tcgen05 tile kernel (head_dim 64 or 128): whether a TMA descriptor can be built for this pool layout, and the launcher
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                           int64_t stride_head);
 // grid_limit > 0 caps the number of CTAs; reset_counter = false joins a grid that is already drawing units

@@ -38,12 +38,12 @@ inline bool tma_encode_pool_map(CUtensorMap* map, bool bf16, const void* pool, i
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The query rows [T][H][128] as a 3-D tensor (column, head, row) read in boxes of 64 columns x 128 rows of one head.
-inline bool tma_encode_q_map(CUtensorMap* map, bool bf16, const void* q, int T, int H) {
+// The query rows [T][H][d] as a 3-D tensor (column, head, row) read in boxes of 64 columns x 128 rows of one head.
+inline bool tma_encode_q_map(CUtensorMap* map, bool bf16, const void* q, int T, int H, int head_dim) {
     EncodeTiledFn fn = tma_encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {128, (cuuint64_t)H, (cuuint64_t)T};
-    const cuuint64_t strides[2] = {128 * 2, (cuuint64_t)H * 128 * 2};
+    const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)H, (cuuint64_t)T};
+    const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)H * head_dim * 2};
     const cuuint32_t box[3] = {64, 1, 128};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(q), dims,

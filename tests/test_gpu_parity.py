@@ -66,6 +66,16 @@ def test_tiny_every_element(cuda_device):
     _check_full(W.tiny(), cuda_device)                       # the full "tiny" configuration
 
 
+def test_head_dim_64_chunks_run_on_the_tcgen05_kernel(cuda_device):
+    """The 64-row chunks of the tiny configuration (8 heads x 64) take the tcgen05 tile kernel, not the mma.sync one."""
+    from paper_2503_18989_b200 import runner
+    sc = W.tiny()
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert sc.cache.head_dim == 64 and ds.info["num_prefill_requests"] == 1 and ds.info["prefill_kernel"] == 1
+    ds.close()
+
+
 def test_llama7b_chunked_reduced(cuda_device):
     _check_full(W.llama7b_chunked(prompt=640, chunk=256, H=4), cuda_device)   # 256, 256, ragged 128
 
