@@ -503,9 +503,26 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         use_tc5 = tc5_layout_supported(p->dtype, p->head_dim, p->num_pages, p->num_kv_heads, cache->stride_page,
                                        cache->stride_token, cache->stride_head);
     p->num_sms = num_sms;
+    // Which tcgen05 tile kernel: the CTA-pair kernel (cta_group::2) shares every K/V tile between the two 128-row halves
+    // of a 256-row unit and is the faster one when every unit fills both halves and there are at least two rounds of
+    // units for the 74 pairs; batches with 64- or 128-row chunks (half of a pair would idle) and small batches keep the
+    // one-CTA kernel.  HAT_PREFILL_KERNEL = tc5 | pair | mma overrides.
     int tile_kernel = use_tc5 ? 1 : 0;
-    if (const char* k = std::getenv("HAT_PREFILL_KERNEL"))
+    if (use_tc5 && p->head_dim == 128) {
+        bool all_wide = true;
+        int64_t wide_tiles = 0;
+        for (int r = 0; r < R; ++r) {
+            const int C = p->chunk_len[r];
+            if (C <= 16) continue;
+            if (C % 256 != 0 && C % 256 <= 128) all_wide = false;
+            wide_tiles += (C + 255) / 256;
+        }
+        if (all_wide && wide_tiles * p->num_heads >= 2 * (int64_t)num_sms) tile_kernel = 3;
+    }
+    if (const char* k = std::getenv("HAT_PREFILL_KERNEL")) {
         if (use_tc5 && p->head_dim == 128 && std::strcmp(k, "pair") == 0) tile_kernel = 3;
+        else if (use_tc5 && std::strcmp(k, "tc5") == 0) tile_kernel = 1;
+    }
     schedule(p, num_sms, tile_kernel);
     // the streaming kernel takes its pages by TMA when a descriptor can be built for the pool layout
     bool stream_tma = true;
