@@ -534,3 +534,44 @@ def test_calls_on_one_plan_from_two_streams_are_kept_in_order(cuda_device):
     assert_parity(out, want[0][0], "two streams out")
     assert_parity(lse, want[0][1], "two streams lse")
     ds.close()
+
+
+# ----------------------------------------------------------------------------
+# both tcgen05 tile kernels, whichever the plan would pick
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("kernel,code", [("pair", 3), ("tc5", 1)])
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_each_tcgen05_tile_kernel_on_every_kind_of_unit(cuda_device, kernel, code, dtype, monkeypatch):
+    """Every element against the oracle with the tile kernel forced: full 256-row units, a 256 + 144 split, units of
+    64 / 128 / 17 rows (half a CTA pair idles, results must not care), prefixes that are not page multiples, an empty
+    prefix, grouped query heads, and streaming-class chunks in the same batch."""
+    from paper_2503_18989_b200 import runner
+    monkeypatch.setenv("HAT_PREFILL_KERNEL", kernel)
+    prefix = [0, 1000, 77, 300, 2049, 5, 640, 33]
+    chunk = [512, 400, 256, 64, 128, 17, 300, 4]
+    sc = _manual(dtype, 2, 128, prefix, chunk, 81, q_group=2)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert ds.info["prefill_kernel"] == code
+    ds.close()
+    _check_full(sc, cuda_device)
+
+
+@pytest.mark.parametrize("kernel", ["pair", "tc5"])
+def test_each_tcgen05_tile_kernel_with_cut_key_ranges_and_sixteen_bit_output(cuda_device, kernel, monkeypatch):
+    from paper_2503_18989_b200 import runner
+    monkeypatch.setenv("HAT_PREFILL_KERNEL", kernel)
+    monkeypatch.setenv("HAT_PREFILL_SPLIT_LEN", "384")          # key ranges of 384: partial rows, merge kernel, ragged last range
+    sc = _manual("bf16", 3, 128, [900, 100, 1500], [512, 256, 300], 83)
+    _check_full(sc, cuda_device)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    ds.attend(fused_append=True)
+    out, lse = ds.results()
+    ds.attend16(fused_append=False)
+    import torch
+    torch.cuda.synchronize()
+    got = W.bits_to_f64(ds.out16.cpu().numpy().view(np.uint16), "bf16").reshape(out.shape)
+    assert ds.canaries_intact()
+    # the 16-bit rows are the fp32 rows rounded once: within half a unit in the last place (2^-8 relative) of them
+    assert np.all(np.abs(got - out) <= np.abs(out) * 2.0 ** -8 + 1e-30)
