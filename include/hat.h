@@ -204,6 +204,35 @@ int hat_kv_append_rope(const hat_cache_desc* cache, const hat_plan* plan, const 
 int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, int interleaved, void* stream);
 
 /*
+ * The projection in front of the attention module with the rotation and the
+ * append in its epilogue (Sec. 2.1: Q = X W_Q, K = X W_K, V = X W_V, and the KV
+ * cache keeps K and V of every token).  For packed row t and output feature f
+ *     y[t][f] = sum_j x[t][j] * w_qkv[f][j]                 (fp32 accumulation)
+ * with the features ordered  num_q_heads heads of q | num_kv_heads heads of k |
+ * num_kv_heads heads of v, head_dim values each.  q and k heads are rotated by
+ * the row's position exactly as hat_rope_q / hat_kv_append_rope do (theta <= 0:
+ * no rotation), every value is rounded to the 16-bit type once, and
+ *     q rows go to q_out[t][h][:]
+ *     k and v rows go to logical token prefix_len[r]+i of request r's cache,
+ *     as hat_kv_append would store them; no other slot of the pools is written.
+ * hat_chunk_attention then takes q_out and no k_new/v_new.
+ *   x          device, [T][hidden], the cache's 16-bit type, 16-byte aligned
+ *   hidden     columns of x and of w_qkv; a multiple of 64
+ *   w_qkv      device, [(num_q_heads + 2 num_kv_heads) * head_dim][hidden]: one
+ *              row per output feature (the paper's W_Q | W_K | W_V, transposed)
+ *   q_out      device, [T][num_q_heads][head_dim], 16-byte aligned
+ *   workspace  device, 256-byte aligned, hat_qkv_workspace_bytes() bytes (the
+ *              cosines and sines of every row); unused when theta <= 0
+ * head_dim 64 or 128.  Nothing is owned or kept by the library.  Errors:
+ * INVALID_ARG, UNSUPPORTED (hidden not a multiple of 64, other head_dim),
+ * WORKSPACE_TOO_SMALL, CUDA; a device-side wait that ran out shows in
+ * hat_last_device_status.
+ */
+int hat_qkv_workspace_bytes(const hat_plan* plan, size_t* out);
+int hat_qkv_rope_append(const hat_cache_desc* cache, const hat_plan* plan, const void* x, int hidden, const void* w_qkv,
+                        void* q_out, float theta, int interleaved, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Chunk attention (Sec. 2.1 self-attention over the KV cache; Sec. 2.1 / 3.3
  * prompt chunks; Sec. 3.4 draft verification).  For packed row t = cu_chunk[r]+i
  * and head h, with g = prefix_len[r]+i and keys/values j = 0..g read through

@@ -634,6 +634,30 @@ int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, in
     return e == cudaSuccess ? HAT_OK : cuda_fail(e);
 }
 
+int hat_qkv_workspace_bytes(const hat_plan* plan, size_t* out) {
+    if (!plan || !out) return HAT_ERR_INVALID_ARG;
+    *out = qkv_workspace_bytes(plan);
+    return HAT_OK;
+}
+
+int hat_qkv_rope_append(const hat_cache_desc* cache, const hat_plan* plan, const void* x, int hidden, const void* w_qkv,
+                        void* q_out, float theta, int interleaved, void* workspace, size_t workspace_bytes, void* stream) {
+    int st = check_call(cache, plan);
+    if (st != HAT_OK) return st;
+    if (theta > 0.f && (!(theta > 1.f) || !std::isfinite(theta))) return HAT_ERR_INVALID_ARG;
+    if (hidden <= 0) return HAT_ERR_INVALID_ARG;
+    if (hidden % 64 != 0 || (plan->head_dim != 64 && plan->head_dim != 128)) return HAT_ERR_UNSUPPORTED;
+    if (plan->total_rows == 0) return HAT_OK;
+    if (!x || !w_qkv || !q_out || !aligned(x, 16) || !aligned(w_qkv, 16) || !aligned(q_out, 16)) return HAT_ERR_INVALID_ARG;
+    if (theta > 0.f) {
+        if (!workspace || !aligned(workspace, 256)) return HAT_ERR_INVALID_ARG;
+        if (workspace_bytes < qkv_workspace_bytes(plan)) return HAT_ERR_WORKSPACE_TOO_SMALL;
+    }
+    cudaError_t e = launch_qkv_gemm(plan, view_of(cache), cache->k_pool, cache->v_pool, x, hidden, w_qkv, q_out, theta,
+                                    interleaved != 0, workspace, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? HAT_OK : cuda_fail(e);
+}
+
 // One attention step; the final rows go to `out` (fp32) or, when out16 is given, to out16 in the cache's 16-bit type.
 static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, const void* q, const void* k_new,
                          const void* v_new, float* out, void* out16, float* lse, float sm_scale, void* workspace,

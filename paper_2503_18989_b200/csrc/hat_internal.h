@@ -113,6 +113,19 @@ __device__ __forceinline__ int hat_in_range(int i, int n, int32_t* status) {
 #define HAT_CHECK(cond, status) do { } while (0)
 #endif
 
+// Rotary position encoding: theta^(-2c/d) for c = 0 .. d/2 - 1, computed on the host in double and passed by value
+struct InvFreq { double f[64]; };
+#ifdef __CUDACC__
+// sine and cosine of position p times one of those factors: the angle is formed and reduced to [-pi, pi] in double,
+// the functions themselves are fp32
+__device__ __forceinline__ void rope_sincos(int p, double inv_freq, float* s, float* c) {
+    const double ang = (double)p * inv_freq;
+    const double turns = rint(ang * 0.15915494309189535);                  // 1 / (2 pi)
+    const double red = fma(-turns, 6.283185307179586, ang) - turns * 2.4492935982947064e-16;
+    sincosf((float)red, s, c);
+}
+#endif
+
 #ifdef __CUDACC__
 // Two fp32 values rounded to nearest into one 32-bit word of the 16-bit output type (low half = first value).
 __device__ __forceinline__ uint32_t pack_out16(float lo, float hi, int bf16) {
@@ -205,6 +218,12 @@ cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStr
 bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                              int64_t stride_head);
 cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+// Q/K/V projection with the rotation and the cache write in its epilogue (tcgen05); theta <= 0: no rotation.
+// `workspace` holds the (cos, sin) table of qkv_workspace_bytes(plan) bytes when theta > 0.
+size_t qkv_workspace_bytes(const hat_plan* plan);
+cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* k_pool, void* v_pool, const void* x,
+                            int hidden, const void* w, void* q_out, float theta, int interleaved, void* workspace,
+                            cudaStream_t stream);
 void count_launch(int n = 1);
 void set_last_cuda_error(int e);   // what hat_last_cuda_error() returns on this thread
 }  // namespace hat

@@ -16,16 +16,6 @@
 namespace hat {
 namespace {
 
-// theta^(-2c/d) for c = 0 .. d/2 - 1, computed on the host in double and passed by value
-struct InvFreq { double f[64]; };
-
-__device__ __forceinline__ void sincos_at(int p, double inv_freq, float* s, float* c) {
-    const double ang = (double)p * inv_freq;
-    const double turns = rint(ang * 0.15915494309189535);                  // 1 / (2 pi)
-    const double red = fma(-turns, 6.283185307179586, ang) - turns * 2.4492935982947064e-16;
-    sincosf((float)red, s, c);
-}
-
 template <bool BF16>
 __device__ __forceinline__ float2 unpack2(uint32_t w) {
     if constexpr (BF16) return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
@@ -58,7 +48,7 @@ rope_kernel(DevicePlan plan, int heads, int d, const __grid_constant__ InvFreq f
     const int vb = interleaved ? 2 * pv + 1 : pv + pairs_vec;
     float sn[8], cs[8];                                                  // pair 8 pv + k of every head
 #pragma unroll
-    for (int k = 0; k < 8; ++k) sincos_at(p, fr.f[8 * pv + k], &sn[k], &cs[k]);
+    for (int k = 0; k < 8; ++k) rope_sincos(p, fr.f[8 * pv + k], &sn[k], &cs[k]);
 
     int64_t pool_base = 0;
     if (to_cache) {

@@ -83,6 +83,20 @@ def normal_bits(n: int, dtype: str, seed: int, threads: int = 8) -> np.ndarray:
     return out
 
 
+def projection_inputs(seed: int, dtype: str, rows: int, hidden: int, features: int):
+    """Layer input x [rows, hidden] ~ N(0,1) and projection weights w [features, hidden] ~ N(0, 1/hidden) (so that
+    the projected values are ~ N(0,1) like the q/k/v of the other workloads), both as uint16 bits."""
+    x = normal_bits(rows * hidden, dtype, seed + 21).reshape(rows, hidden)
+    g = np.random.Generator(np.random.PCG64(seed + 22))
+    w = np.empty((features, hidden), dtype=np.uint16)
+    inv = np.float32(1.0 / np.sqrt(hidden))
+    step = max(1, (1 << 24) // hidden)
+    for lo in range(0, features, step):
+        hi = min(features, lo + step)
+        w[lo:hi] = f32_to_bits(g.standard_normal((hi - lo, hidden), dtype=np.float32) * inv, dtype)
+    return x, w
+
+
 # --------------------------------------------------------------------------
 # Descriptors
 # --------------------------------------------------------------------------

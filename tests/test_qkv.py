@@ -75,3 +75,131 @@ def test_projection_is_additive_in_the_weights_and_rejects_bad_shapes():
         QO.project(xb, b1[:, :15], "fp16")
     with pytest.raises(ValueError):
         QO.qkv_rope(xb, b1, np.zeros(5, np.int64), "fp16", 2, 1, 4)            # 12 rows are not (2 + 2) * 4
+
+
+# ----------------------------------------------------------------------------
+# GPU parity
+# ----------------------------------------------------------------------------
+def _assert_projected(got_bits, want_bits, dtype, what, exact_share):
+    """fp32 accumulation on the tensor cores, fp32 rotation, one rounding, against float64 rounded once: the same bits
+    nearly everywhere; elsewhere within one unit in the last place plus the accumulation error (hidden <= 5120 terms
+    of magnitude <= 1, each step rounded to 2^-23 of a partial sum of a few units: below 2e-4)."""
+    got, want = W.bits_to_f64(got_bits, dtype), W.bits_to_f64(want_bits, dtype)
+    assert np.isfinite(got).all(), what
+    ulp = np.abs(want) * (2.0 ** -10 if dtype == "fp16" else 2.0 ** -7)
+    worst = float(np.max(np.abs(got - want) - ulp))
+    assert worst <= 2e-4, (what, worst)
+    share = float(np.mean(got_bits == want_bits))
+    assert share > exact_share, (what, share)
+
+
+def _run_projection(cuda_device, dtype, d, hq, hkv, hidden, prefix, chunk, theta, interleaved, seed=11):
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    rng = np.random.Generator(np.random.PCG64(seed))
+    table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=4)
+    st = W._make_step(500 + seed, dtype, hkv, d, prefix, chunk, table, q_heads=hq)
+    sc = W._scenario("qkv", dtype, hkv, d, "paged", num_pages, [st], 500 + seed)
+    T = st.total_rows
+    feats = (hq + 2 * hkv) * d
+    xb, wb = W.projection_inputs(700 + seed, dtype, T, hidden, feats)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    x_dev = runner._dev_u16(xb, cuda_device)
+    w_dev = runner._dev_u16(wb, cuda_device)
+    g_q = runner._Guarded((T, hq, d), torch.int16, -1, cuda_device)
+    ws_bytes = B.hat_qkv_workspace_bytes(ds.plan)
+    g_ws = runner._Guarded((max(ws_bytes, 256),), torch.uint8, None, cuda_device)
+    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, g_q.view, theta, interleaved, g_ws.view, ws_bytes)
+    torch.cuda.synchronize()
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    assert g_q.intact() and g_ws.intact(), "a canary zone around q_out / workspace was overwritten"
+    got_q = g_q.view.cpu().numpy().view(np.uint16).reshape(T, hq, d)
+    gk, gv = cache.pools_to_host()
+    return sc, st, ds, cache, xb, wb, got_q, gk, gv
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype,d,hq,hkv,hidden,theta,interleaved", [
+    ("fp16", 128, 4, 2, 320, 10000.0, False),      # 4 feature tiles, 5 stages of the hidden dimension (the ring wraps)
+    ("bf16", 128, 2, 2, 64, 10000.0, True),        # one stage per tile
+    ("bf16", 64, 6, 3, 128, 10000.0, True),        # four heads per feature tile
+    ("fp16", 64, 3, 1, 192, 500000.0, False),      # 320 features: the second feature tile is partly empty
+    ("fp16", 128, 3, 1, 128, 0.0, False),          # no rotation; 5 heads: the last tile holds one
+])
+def test_projection_kernel_rotates_and_appends(cuda_device, dtype, d, hq, hkv, hidden, theta, interleaved):
+    """hat_qkv_rope_append against the float64 projection, rotation and append: q rows, the written slots of both
+    pools (and nothing but them), over several row tiles with a ragged last one."""
+    prefix, chunk = [0, 37, 1000, 4090, 8000, 250], [5, 130, 16, 200, 8, 0]
+    sc, st, ds, cache, xb, wb, got_q, gk, gv = _run_projection(cuda_device, dtype, d, hq, hkv, hidden, prefix, chunk,
+                                                               theta, interleaved)
+    pos = R.positions(st)
+    want_q, want_k, want_v = QO.qkv_rope(xb, wb, pos, dtype, hq, hkv, d, theta if theta > 0 else None, interleaved)
+    _assert_projected(got_q, want_q, dtype, "q rows", 0.97)
+    ref = types.SimpleNamespace(**{**st.__dict__, "k_new": want_k, "v_new": want_v})
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(sc.cache, kp, vp, ref)
+    # slots of the chunk rows: found by appending a marker pattern through the oracle
+    mark = types.SimpleNamespace(**{**st.__dict__, "k_new": np.full_like(want_k, 0xFFFF), "v_new": np.full_like(want_v, 0xFFFF)})
+    mk, mv = np.zeros_like(kp), np.zeros_like(vp)
+    O.kv_append(sc.cache, mk, mv, mark)
+    written = mk == 0xFFFF
+    assert written.sum() == want_k.size
+    assert np.array_equal(gk[~written], sc.k_pool[~written]), "a K slot outside the chunk was written"
+    assert np.array_equal(gv[~written], sc.v_pool[~written]), "a V slot outside the chunk was written"
+    _assert_projected(gk[written], kp[written], dtype, "K in the pool", 0.97)
+    _assert_projected(gv[written], vp[written], dtype, "V in the pool", 0.97)
+    ds.close()
+
+
+@pytest.mark.gpu
+def test_projection_then_attention_matches_the_oracle_step(cuda_device):
+    """The whole layer front: projection kernel, then hat_chunk_attention on its q rows and the cache it wrote, against
+    the oracle's attention over the oracle's own projected, rotated and appended rows."""
+    import torch
+    from paper_2503_18989_b200 import binding as B
+    from common import assert_parity
+    dtype, d, hq, hkv, hidden = "bf16", 128, 4, 2, 256
+    prefix, chunk = [0, 300, 2000], [256, 4, 70]
+    sc, st, ds, cache, xb, wb, got_q, gk, gv = _run_projection(cuda_device, dtype, d, hq, hkv, hidden, prefix, chunk,
+                                                               10000.0, False, seed=12)
+    q_dev = torch.from_numpy(got_q.view(np.int16)).to(cuda_device)
+    B.hat_chunk_attention(cache.desc, ds.plan, q_dev, None, None, ds.out, ds.lse, 0.0, ds.workspace, ds.workspace_bytes)
+    go, gl = ds.results()
+    want_q, want_k, want_v = QO.qkv_rope(xb, wb, R.positions(st), dtype, hq, hkv, d)
+    ref = types.SimpleNamespace(**{**st.__dict__, "q": want_q, "k_new": want_k, "v_new": want_v})
+    kp, vp = sc.k_pool.copy(), sc.v_pool.copy()
+    O.kv_append(sc.cache, kp, vp, ref)
+    wo, wl = O.chunk_attention(sc.cache, kp, vp, ref)
+    assert_parity(go, wo, "layer front out")
+    assert_parity(gl, wl, "layer front lse")
+    ds.close()
+
+
+@pytest.mark.gpu
+def test_projection_kernel_rejects_what_it_cannot_run(cuda_device):
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    rng = np.random.Generator(np.random.PCG64(3))
+    table, num_pages = W._place_pages(rng, np.asarray([20]), slack_pages=1)
+    st = W._make_step(1, "fp16", 1, 128, [4], [16], table, q_heads=1)
+    sc = W._scenario("qkv", "fp16", 1, 128, "paged", num_pages, [st], 1)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    x = torch.zeros(16 * 96, dtype=torch.int16, device=cuda_device)
+    w = torch.zeros(384 * 96, dtype=torch.int16, device=cuda_device)
+    q = torch.zeros(16 * 128, dtype=torch.int16, device=cuda_device)
+    ws = torch.zeros(B.hat_qkv_workspace_bytes(ds.plan), dtype=torch.uint8, device=cuda_device)
+    L = B.lib()
+    import ctypes as C
+    def call(hidden, theta, ws_t, ws_n, xp=x):
+        return L.hat_qkv_rope_append(C.byref(cache.desc), B._h(ds.plan),
+                                     B._ptr(xp), hidden, B._ptr(w), B._ptr(q), C.c_float(theta), 0, B._ptr(ws_t), ws_n, None)
+    assert call(96, 10000.0, ws, ws.numel()) == B.HAT_ERR_UNSUPPORTED            # hidden not a multiple of 64
+    assert call(64, 0.5, ws, ws.numel()) == B.HAT_ERR_INVALID_ARG                # a base in (0, 1]
+    assert call(64, 10000.0, None, 0) == B.HAT_ERR_INVALID_ARG                   # rotation without its table
+    assert call(64, 10000.0, ws, 8) == B.HAT_ERR_WORKSPACE_TOO_SMALL
+    assert call(64, 10000.0, ws, ws.numel(), xp=None) == B.HAT_ERR_INVALID_ARG
+    assert call(64, 10000.0, ws, ws.numel()) == B.HAT_OK
+    torch.cuda.synchronize()
+    ds.close()
