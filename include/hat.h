@@ -221,16 +221,12 @@ int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, in
  *   w_qkv      device, [(num_q_heads + 2 num_kv_heads) * head_dim][hidden]: one
  *              row per output feature (the paper's W_Q | W_K | W_V, transposed)
  *   q_out      device, [T][num_q_heads][head_dim], 16-byte aligned
- *   workspace  device, 256-byte aligned, hat_qkv_workspace_bytes() bytes (the
- *              cosines and sines of every row); unused when theta <= 0
  * head_dim 64 or 128.  Nothing is owned or kept by the library.  Errors:
- * INVALID_ARG, UNSUPPORTED (hidden not a multiple of 64, other head_dim),
- * WORKSPACE_TOO_SMALL, CUDA; a device-side wait that ran out shows in
- * hat_last_device_status.
+ * INVALID_ARG, UNSUPPORTED (hidden not a multiple of 64, other head_dim), CUDA;
+ * a device-side wait that ran out shows in hat_last_device_status.
  */
-int hat_qkv_workspace_bytes(const hat_plan* plan, size_t* out);
 int hat_qkv_rope_append(const hat_cache_desc* cache, const hat_plan* plan, const void* x, int hidden, const void* w_qkv,
-                        void* q_out, float theta, int interleaved, void* workspace, size_t workspace_bytes, void* stream);
+                        void* q_out, float theta, int interleaved, void* stream);
 
 /*
  * Chunk attention (Sec. 2.1 self-attention over the KV cache; Sec. 2.1 / 3.3

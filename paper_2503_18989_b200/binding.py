@@ -34,7 +34,7 @@ DTYPE_CODE = {"fp16": HAT_DTYPE_FP16, "bf16": HAT_DTYPE_BF16}
 EXPORTS = [
     "hat_status_string", "hat_version", "hat_last_cuda_error", "hat_launch_count",
     "hat_plan_create", "hat_plan_get_info", "hat_plan_workspace_bytes", "hat_plan_destroy",
-    "hat_kv_append", "hat_kv_append_rope", "hat_rope_q", "hat_qkv_workspace_bytes", "hat_qkv_rope_append", "hat_chunk_attention", "hat_chunk_attention_out16",
+    "hat_kv_append", "hat_kv_append_rope", "hat_rope_q", "hat_qkv_rope_append", "hat_chunk_attention", "hat_chunk_attention_out16",
     "hat_plan_staging_bytes",
     "hat_chunk_attention_host",
     "hat_last_device_status", "hat_plan_enable_timing", "hat_plan_read_timing",
@@ -117,10 +117,8 @@ def lib() -> C.CDLL:
         L.hat_kv_append_rope.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, C.c_float, i32, vp]
         L.hat_rope_q.restype = i32
         L.hat_rope_q.argtypes = [vp, vp, vp, C.c_float, i32, vp]
-        L.hat_qkv_workspace_bytes.restype = i32
-        L.hat_qkv_workspace_bytes.argtypes = [vp, C.POINTER(sz)]
         L.hat_qkv_rope_append.restype = i32
-        L.hat_qkv_rope_append.argtypes = [C.POINTER(hat_cache_desc), vp, vp, i32, vp, vp, C.c_float, i32, vp, sz, vp]
+        L.hat_qkv_rope_append.argtypes = [C.POINTER(hat_cache_desc), vp, vp, i32, vp, vp, C.c_float, i32, vp]
         L.hat_chunk_attention.restype = i32
         L.hat_chunk_attention.argtypes = [C.POINTER(hat_cache_desc), vp, vp, vp, vp, vp, vp, C.c_float, vp, sz, vp]
         L.hat_chunk_attention_out16.restype = i32
@@ -278,17 +276,10 @@ def hat_rope_q(plan, q, q_out, theta: float = 10000.0, interleaved: bool = False
            "hat_rope_q")
 
 
-def hat_qkv_workspace_bytes(plan) -> int:
-    n = C.c_size_t(0)
-    _check(lib().hat_qkv_workspace_bytes(_h(plan), C.byref(n)), "hat_qkv_workspace_bytes")
-    return int(n.value)
-
-
 def hat_qkv_rope_append(cache: hat_cache_desc, plan, x, hidden: int, w_qkv, q_out, theta: float = 10000.0,
-                        interleaved: bool = False, workspace=None, workspace_bytes: int = 0, stream: int = 0) -> None:
+                        interleaved: bool = False, stream: int = 0) -> None:
     _check(lib().hat_qkv_rope_append(C.byref(cache), _h(plan), _ptr(x), int(hidden), _ptr(w_qkv), _ptr(q_out),
-                                     C.c_float(theta), int(bool(interleaved)), _ptr(workspace), int(workspace_bytes),
-                                     stream or None), "hat_qkv_rope_append")
+                                     C.c_float(theta), int(bool(interleaved)), stream or None), "hat_qkv_rope_append")
 
 
 def hat_chunk_attention(cache: hat_cache_desc, plan, q, k_new, v_new, out, lse, sm_scale: float = 0.0,

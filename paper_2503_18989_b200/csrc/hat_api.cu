@@ -332,11 +332,15 @@ static int upload(hat_plan* p) {
 
     cudaError_t e = cudaGetDevice(&p->device);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaMalloc(&p->dev_blob, blob.size());
+    // behind the arrays: room for the (cos, sin) table of the projection epilogue, filled on the device when first used
+    const size_t o_table = (blob.size() + 255) / 256 * 256;
+    const size_t table_bytes = (size_t)p->total_rows * (p->head_dim / 2) * sizeof(float2);
+    e = cudaMalloc(&p->dev_blob, o_table + std::max<size_t>(table_bytes, 16));
     if (e != cudaSuccess) { p->dev_blob = nullptr; return cuda_fail(e); }
     e = cudaMemcpy(p->dev_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) return cuda_fail(e);
     char* base = static_cast<char*>(p->dev_blob);
+    p->rope_table = reinterpret_cast<float2*>(base + o_table);
     DevicePlan& d = p->dev;
     d.cu_chunk = reinterpret_cast<const int32_t*>(base + o_cu);
     d.prefix_len = reinterpret_cast<const int32_t*>(base + o_pl);
@@ -459,6 +463,10 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     p->num_verify_merge_rows = 0;
     p->ev_verify = nullptr;
     p->ev_done = nullptr;
+    p->ev_table = nullptr;
+    p->rope_table = nullptr;
+    p->rope_theta = 0.f;
+    p->table_stream = nullptr;
     p->last_stream = nullptr;
     p->has_last = false;
     p->side_sms = 0;
@@ -546,6 +554,8 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
         if (ee != cudaSuccess) { p->ev_verify = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
         ee = cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming);
         if (ee != cudaSuccess) { p->ev_done = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
+        ee = cudaEventCreateWithFlags(&p->ev_table, cudaEventDisableTiming);
+        if (ee != cudaSuccess) { p->ev_table = nullptr; hat_plan_destroy(p); return cuda_fail(ee); }
         // Optional throughput mode for a mixed batch on the tcgen05 path (HAT_SIDE_SMS = n > 0): see the launch
         // sequence.  Off by default: it finishes the whole step sooner but the decode-phase rows later.  The side
         // stream has the highest priority so that the tile CTAs are placed before the streaming kernel's many small
@@ -589,6 +599,7 @@ int hat_plan_destroy(hat_plan* plan) {
     }
     if (plan->ev_verify) cudaEventDestroy(plan->ev_verify);
     if (plan->ev_done) cudaEventDestroy(plan->ev_done);
+    if (plan->ev_table) cudaEventDestroy(plan->ev_table);
     if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
     if (plan->ev_join) cudaEventDestroy(plan->ev_join);
     if (plan->aux_stream) cudaStreamDestroy(plan->aux_stream);
@@ -634,14 +645,8 @@ int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, in
     return e == cudaSuccess ? HAT_OK : cuda_fail(e);
 }
 
-int hat_qkv_workspace_bytes(const hat_plan* plan, size_t* out) {
-    if (!plan || !out) return HAT_ERR_INVALID_ARG;
-    *out = qkv_workspace_bytes(plan);
-    return HAT_OK;
-}
-
 int hat_qkv_rope_append(const hat_cache_desc* cache, const hat_plan* plan, const void* x, int hidden, const void* w_qkv,
-                        void* q_out, float theta, int interleaved, void* workspace, size_t workspace_bytes, void* stream) {
+                        void* q_out, float theta, int interleaved, void* stream) {
     int st = check_call(cache, plan);
     if (st != HAT_OK) return st;
     if (theta > 0.f && (!(theta > 1.f) || !std::isfinite(theta))) return HAT_ERR_INVALID_ARG;
@@ -649,12 +654,8 @@ int hat_qkv_rope_append(const hat_cache_desc* cache, const hat_plan* plan, const
     if (hidden % 64 != 0 || (plan->head_dim != 64 && plan->head_dim != 128)) return HAT_ERR_UNSUPPORTED;
     if (plan->total_rows == 0) return HAT_OK;
     if (!x || !w_qkv || !q_out || !aligned(x, 16) || !aligned(w_qkv, 16) || !aligned(q_out, 16)) return HAT_ERR_INVALID_ARG;
-    if (theta > 0.f) {
-        if (!workspace || !aligned(workspace, 256)) return HAT_ERR_INVALID_ARG;
-        if (workspace_bytes < qkv_workspace_bytes(plan)) return HAT_ERR_WORKSPACE_TOO_SMALL;
-    }
     cudaError_t e = launch_qkv_gemm(plan, view_of(cache), cache->k_pool, cache->v_pool, x, hidden, w_qkv, q_out, theta,
-                                    interleaved != 0, workspace, static_cast<cudaStream_t>(stream));
+                                    interleaved != 0, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? HAT_OK : cuda_fail(e);
 }
 

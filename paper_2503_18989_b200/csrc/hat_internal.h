@@ -192,6 +192,12 @@ struct hat_plan {
     long long wait_cycles;      // bound of device-side waits (default: about a second)
     int withhold_next;          // self test of the bounded waits: applies to the next attention call only
     hat::MapCache maps;         // see MapCache (updated through const_cast by the launchers: one call at a time per plan)
+    // rotary position encoding in the projection epilogue: (cos, sin) of every row and pair for base rope_theta
+    // (0: not filled yet), inside dev_blob; ev_table orders calls on other streams behind the kernel that filled it
+    float2* rope_table;
+    float rope_theta;
+    cudaStream_t table_stream;
+    cudaEvent_t ev_table;
     void* dev_blob;             // one allocation holding every device array
     hat::DevicePlan dev;
 };
@@ -218,12 +224,9 @@ cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStr
 bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                              int64_t stride_head);
 cudaError_t launch_attn_stream(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
-// Q/K/V projection with the rotation and the cache write in its epilogue (tcgen05); theta <= 0: no rotation.
-// `workspace` holds the (cos, sin) table of qkv_workspace_bytes(plan) bytes when theta > 0.
-size_t qkv_workspace_bytes(const hat_plan* plan);
+// Q/K/V projection with the rotation and the cache write in its epilogue (tcgen05); theta <= 0: no rotation
 cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* k_pool, void* v_pool, const void* x,
-                            int hidden, const void* w, void* q_out, float theta, int interleaved, void* workspace,
-                            cudaStream_t stream);
+                            int hidden, const void* w, void* q_out, float theta, int interleaved, cudaStream_t stream);
 void count_launch(int n = 1);
 void set_last_cuda_error(int e);   // what hat_last_cuda_error() returns on this thread
 }  // namespace hat

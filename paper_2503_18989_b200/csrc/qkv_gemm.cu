@@ -4,20 +4,28 @@
 //
 //   y[t][f] = sum_j x[t][j] w[f][j]        x [T][hidden], w [(Hq + 2 Hkv) d][hidden] (one row per output feature),
 //                                          features ordered q heads | k heads | v heads
-// Persistent kernel, one CTA per SM, output tiles of 128 rows x 256 features (two heads of 128 or four of 64), drawn
-// in a fixed order with the row tile running fastest: the CTAs of one round share a strip of w, which then crosses
-// HBM once, and x (much smaller) stays in L2.  Roles:
-//   warp 0      TMA producer: per 64 columns of the hidden dimension one box of x (128 rows) and one of w (256 rows),
-//               128-byte swizzle, into a four-stage ring
-//   warp 1      one thread issues tcgen05.mma (M 128, N 256, K 16; four per stage) into one of two 256-column
-//               accumulators in TMEM; tcgen05.commit frees the stage and, after the last stage of a tile, hands the
-//               accumulator to the epilogue.  Owns the TMEM allocation
+// Persistent kernel, output tiles of 256 features (two heads of 128 or four of 64), drawn in a fixed order with the row
+// tile running fastest: the CTAs of one round share a strip of w, which then crosses HBM once, and x (much smaller)
+// stays in L2.  Two forms:
+//   PAIR   clusters of two CTAs, tcgen05.mma.cta_group::2 with M = 256: each CTA stages its own 128 rows of x and
+//          HALF of the 256 rows of w (32 KiB per 64 columns of the hidden dimension and CTA, six stages).  What bounds
+//          this GEMM on 148 SMs is the path from L2 into shared memory, and a pair moves 2/3 of the bytes per flop that
+//          two single CTAs do
+//   single one CTA per tile of 128 rows (48 KiB per stage, four stages): batches of at most 128 rows, which would leave
+//          half of a pair idle
+// Roles (per CTA):
+//   warp 0      TMA producer: per 64 columns of the hidden dimension one box of x and one of w, 128-byte swizzle
+//   warp 1      CTA 0 of a pair (or the single CTA): one thread issues tcgen05.mma (four per stage) into one of two
+//               256-column accumulators in TMEM; tcgen05.commit frees the stage (in both CTAs) and, after the last
+//               stage of a tile, hands the accumulator to the epilogue warps.  CTA 1: one thread forwards "my half of
+//               this stage has landed" to CTA 0's barrier.  The warp owns the TMEM allocation
 //   warps 2-5   epilogue, thread = output row = TMEM lane: reads the accumulator 32 columns at a time, rotates q and k
-//               heads with the (cos, sin) pairs of the row's position (a table filled by a small kernel in front, the
-//               same double-precision angle reduction as the rotating append), rounds to the 16-bit type once and
-//               stores q rows packed and k / v rows at their slot of the pools; the other accumulator is being
-//               filled meanwhile
-// Every wait is bounded; a wait that gives up sets bit 0 of the plan's status word and the CTA winds down normally.
+//               heads with the (cos, sin) of the row's position (a table kept with the plan, filled once per plan and
+//               base by a small kernel with the same double-precision angle reduction as the rotating append), rounds
+//               to the 16-bit type once and stores q rows packed and k / v rows at their slot of the pools; the other
+//               accumulator is being filled meanwhile
+// Every wait is bounded; a wait that gives up sets bit 0 of the plan's status word, tells the other CTA of the pair, and
+// the CTA winds down normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -34,22 +42,27 @@ namespace {
 using namespace tc5;
 
 constexpr int kTileM = 128, kTileN = 256, kTileK = 64;
-constexpr int kStages = 4;
-constexpr uint32_t kABytes = kTileM * kTileK * 2;        // 16 KiB
-constexpr uint32_t kBBytes = kTileN * kTileK * 2;        // 32 KiB
-constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kABytes = kTileM * kTileK * 2;        // 16 KiB: 128 rows of x
 constexpr int kThreads = 192;
+constexpr int kMaxStages = 6;
+
+template <bool PAIR> struct Geo {
+    static constexpr int kStages = PAIR ? 6 : 4;
+    static constexpr int kBRows = PAIR ? kTileN / 2 : kTileN;            // rows of w one CTA stages
+    static constexpr uint32_t kBBytes = kBRows * kTileK * 2;
+    static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+};
 
 struct __align__(8) Barriers {
-    uint64_t full[kStages], empty[kStages];
+    uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t acc_full[2], acc_empty[2];
     uint64_t drain;
     long long wait_cycles;
     uint32_t tmem_base;
     volatile int abort_flag;
 };
-constexpr uint32_t kSmemBytes = 1024 + kStages * kStageBytes + sizeof(Barriers);
-static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
+template <bool PAIR> constexpr uint32_t smem_bytes() { return 1024 + Geo<PAIR>::kStages * Geo<PAIR>::kStageBytes + sizeof(Barriers); }
+static_assert(smem_bytes<true>() <= 227 * 1024 && smem_bytes<false>() <= 227 * 1024, "shared memory of one CTA");
 
 struct QkvArgs {
     DevicePlan plan;
@@ -57,20 +70,28 @@ struct QkvArgs {
     void* k_pool;
     void* v_pool;
     void* q_out;              // [T][Hq][d]
-    const float2* trig;       // [T][d/2] (cos, sin), or null: no rotation
+    const float2* trig;       // [T][d/2] (cos, sin), or null: q and k are stored as projected
     int hidden, head_dim, interleaved;
-    int m_tiles, n_tiles;
+    int m_tiles, n_tiles;     // row tiles (of 256 rows for pairs, else 128) and feature tiles
     long long wait_cycles;
 };
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* b, int32_t* status) {
+struct Ctx {
+    Barriers* bars;
+    int32_t* status;
+    uint32_t peer_abort;      // shared::cluster address of the other CTA's abort flag (pairs)
+    bool pair;
+};
+
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const Ctx& cx) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try(bar, parity)) {
-        if (b->abort_flag) return false;
-        if (clock64() - t0 > b->wait_cycles) {
-            b->abort_flag = 1;
-            atomicOr(status, 1);
+        if (cx.bars->abort_flag) return false;
+        if (clock64() - t0 > cx.bars->wait_cycles) {
+            cx.bars->abort_flag = 1;
+            if (cx.pair) st_cluster_b32(cx.peer_abort, 1u);
+            atomicOr(cx.status, 1);
             return false;
         }
     }
@@ -104,21 +125,121 @@ __global__ void __launch_bounds__(256) rope_table_kernel(DevicePlan plan, int ha
     trig[idx] = make_float2(co, s);
 }
 
+// One output row of one tile: the thread's TMEM lane of the accumulator at `acc`, packed row t, feature tile n.
 template <bool BF16>
+__device__ __forceinline__ void epilogue_row(const QkvArgs& a, uint32_t acc, int t, int n, int32_t* status) {
+    const int d = a.head_dim, half = d / 2;
+    const int Hq = a.plan.num_heads, Hkv = a.plan.num_kv_heads;
+    const bool valid = t < a.plan.total_rows;
+    int64_t pool_off = 0;                                  // element offset of (page, slot) in the pools
+    const float2* trig = nullptr;
+    if (valid) {
+        const int r = a.plan.row_req[t];
+        const int p = a.plan.prefix_len[r] + (t - a.plan.cu_chunk[r]);
+        const int page = HAT_IN_RANGE(__ldg(a.plan.block_table + (int64_t)r * a.plan.max_pages +
+                                            HAT_IN_RANGE(p / kPageSize, a.plan.max_pages, status)),
+                                      a.plan.num_pages, status);
+        pool_off = (int64_t)page * a.cache.stride_page + (int64_t)(p % kPageSize) * a.cache.stride_token;
+        if (a.trig) trig = a.trig + (int64_t)t * half;
+    }
+    const int h_first = (n * kTileN) / d;                  // first head of this tile
+    const int h_count = min(kTileN / d, Hq + 2 * Hkv - h_first);
+    for (int hi = 0; hi < h_count; ++hi) {
+        const int hh = h_first + hi;
+        // where the head's d values of this row go
+        unsigned char* dst;
+        bool rot = a.trig != nullptr;
+        if (hh < Hq) {
+            dst = static_cast<unsigned char*>(a.q_out) + ((int64_t)t * Hq + hh) * d * 2;
+        } else if (hh < Hq + Hkv) {
+            dst = static_cast<unsigned char*>(a.k_pool) + (pool_off + (int64_t)(hh - Hq) * a.cache.stride_head) * 2;
+        } else {
+            dst = static_cast<unsigned char*>(a.v_pool) + (pool_off + (int64_t)(hh - Hq - Hkv) * a.cache.stride_head) * 2;
+            rot = false;
+        }
+        const uint32_t col = acc + hi * d;
+        if (!rot) {
+            for (int c0 = 0; c0 < d; c0 += 32) {
+                float v[32];
+                tmem_ld32(col + c0, reinterpret_cast<uint32_t*>(v));
+                tmem_ld_wait();
+                if (valid) store32<BF16>(dst + c0 * 2, v);
+            }
+        } else if (a.interleaved) {
+            // pairs (x[2c], x[2c+1]): 32 columns hold pairs c0/2 .. c0/2 + 15
+            for (int c0 = 0; c0 < d; c0 += 32) {
+                float v[32];
+                tmem_ld32(col + c0, reinterpret_cast<uint32_t*>(v));
+                tmem_ld_wait();
+                if (valid) {
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        const float4 cs = __ldg(reinterpret_cast<const float4*>(trig + c0 / 2 + i));   // two (cos, sin)
+                        const float lo0 = v[2 * i], hi0 = v[2 * i + 1], lo1 = v[2 * i + 2], hi1 = v[2 * i + 3];
+                        v[2 * i] = lo0 * cs.x - hi0 * cs.y;
+                        v[2 * i + 1] = hi0 * cs.x + lo0 * cs.y;
+                        v[2 * i + 2] = lo1 * cs.z - hi1 * cs.w;
+                        v[2 * i + 3] = hi1 * cs.z + lo1 * cs.w;
+                    }
+                    store32<BF16>(dst + c0 * 2, v);
+                }
+            }
+        } else {
+            // pairs (x[c], x[c + d/2]): 32 columns of the low half with their partners of the high half
+            for (int c0 = 0; c0 < half; c0 += 32) {
+                float lo[32], hv[32];
+                tmem_ld32(col + c0, reinterpret_cast<uint32_t*>(lo));
+                tmem_ld32(col + half + c0, reinterpret_cast<uint32_t*>(hv));
+                tmem_ld_wait();
+                if (valid) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float4 cs = __ldg(reinterpret_cast<const float4*>(trig + c0 + i));
+                        const float l0 = lo[i], h0 = hv[i], l1 = lo[i + 1], h1 = hv[i + 1];
+                        lo[i] = l0 * cs.x - h0 * cs.y;
+                        hv[i] = h0 * cs.x + l0 * cs.y;
+                        lo[i + 1] = l1 * cs.z - h1 * cs.w;
+                        hv[i + 1] = h1 * cs.z + l1 * cs.w;
+                    }
+                    store32<BF16>(dst + c0 * 2, lo);
+                    store32<BF16>(dst + (half + c0) * 2, hv);
+                }
+            }
+        }
+    }
+}
+
+template <bool BF16, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUtensorMap map_x,
                 const __grid_constant__ CUtensorMap map_w) {
+    using G = Geo<PAIR>;
+    constexpr int kStages = G::kStages;
     extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment for the swizzle pattern; both CTAs of a pair get the same offsets (one descriptor serves both)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    Barriers* bars = reinterpret_cast<Barriers*>(smem + kStages * kStageBytes);
+    Barriers* bars = reinterpret_cast<Barriers*>(smem + kStages * G::kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int32_t* status = a.plan.status;
+    uint32_t rank = 0;                                          // 0: the CTA whose thread issues the MMAs
+    if constexpr (PAIR) rank = cluster_ctarank();
+    Ctx cx;
+    cx.bars = bars;
+    cx.status = a.plan.status;
+    cx.pair = PAIR;
+    cx.peer_abort = 0;
+    if constexpr (PAIR) cx.peer_abort = map_to_cta(smem_u32(const_cast<int*>(&bars->abort_flag)), rank ^ 1u);
     const int k_steps = a.hidden / kTileK;
     const int total_tiles = a.m_tiles * a.n_tiles;
+    const int first_tile = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&bars->acc_full[s], 1); mbar_init(&bars->acc_empty[s], 4); }
+        const uint32_t fwd = (PAIR && rank == 0) ? 2u : 1u;     // CTA 0's "full" barriers also take CTA 1's forwarded arrival
+        for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], fwd); mbar_init(&bars->empty[s], 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->acc_full[s], 1);
+            mbar_init(&bars->acc_empty[s], PAIR ? 8 : 4);       // one arrival per epilogue warp (of both CTAs)
+        }
         mbar_init(&bars->drain, 1);
         bars->abort_flag = 0;
         bars->wait_cycles = a.wait_cycles;
@@ -126,11 +247,21 @@ qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUten
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;\n" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+        if constexpr (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;\n" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;\n" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;\n" ::"r"(smem_u32(&bars->tmem_base)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) {
+        // the other CTA's barriers must be initialised before anything arrives on them
+        cluster_arrive();
+        cluster_wait();
+    }
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
@@ -139,16 +270,18 @@ qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUten
         if (lane == 0) {
             bool ok = true;
             int it = 0;                                        // stages issued so far, over all tiles
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
                 const int m = tile % a.m_tiles, n = tile / a.m_tiles;
+                const int x_row = PAIR ? m * 2 * kTileM + (int)rank * kTileM : m * kTileM;
+                const int w_row = n * kTileN + (int)rank * G::kBRows;
                 for (int ks = 0; ks < k_steps; ++ks, ++it) {
                     const int s = it % kStages;
-                    if (it >= kStages) ok = mbar_wait(&bars->empty[s], ((it / kStages) & 1) ^ 1, bars, status);
+                    if (it >= kStages) ok = mbar_wait(&bars->empty[s], ((it / kStages) & 1) ^ 1, cx);
                     if (!ok) break;
-                    const uint32_t dst = smem_u32(smem) + s * kStageBytes;
-                    mbar_expect_tx(&bars->full[s], kStageBytes);
-                    tma_load_2d(dst, &map_x, ks * kTileK, m * kTileM, &bars->full[s]);
-                    tma_load_2d(dst + kABytes, &map_w, ks * kTileK, n * kTileN, &bars->full[s]);
+                    const uint32_t dst = smem_u32(smem) + s * G::kStageBytes;
+                    mbar_expect_tx(&bars->full[s], G::kStageBytes);
+                    tma_load_2d(dst, &map_x, ks * kTileK, x_row, &bars->full[s]);
+                    tma_load_2d(dst + kABytes, &map_w, ks * kTileK, w_row, &bars->full[s]);
                 }
             }
             if (!ok) {
@@ -158,38 +291,59 @@ qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUten
             }
         }
         __syncwarp();
+    } else if (warp == 1 && rank != 0) {
+        // ------------------------------------------------------------------ CTA 1: forward "landed" to CTA 0's barriers
+        if constexpr (PAIR) {
+            if (lane == 0) {
+                bool ok = true;
+                int it = 0;
+                for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+                    for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                        const int s = it % kStages;
+                        ok = mbar_wait(&bars->full[s], (it / kStages) & 1, cx);
+                        if (!ok) break;
+                        mbar_arrive_remote(map_to_cta(smem_u32(&bars->full[s]), 0u));
+                    }
+                }
+            }
+            __syncwarp();
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (one thread)
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BF16 ? 1u : 0u, 0, kTileM, kTileN);     // x (K-major) x w (K-major)
+            constexpr uint32_t idesc = make_idesc(BF16 ? 1u : 0u, 0, PAIR ? 2 * kTileM : kTileM, kTileN);   // x (K-major) x w (K-major)
             const uint64_t a_desc0 = smem_desc(smem_u32(smem), 16, 1024);
             const uint64_t b_desc0 = smem_desc(smem_u32(smem) + kABytes, 16, 1024);
+            auto commit = [&](uint64_t* bar) { if constexpr (PAIR) tc_commit_pair(bar); else tc_commit(bar); };
             bool ok = true;
             int it = 0, n_done = 0;                            // stages consumed, tiles issued
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++n_done) {
+            for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++n_done) {
                 const int buf = n_done & 1;
                 if (n_done >= 2) {
-                    // the epilogue has read the tile before last out of this accumulator
-                    ok = mbar_wait(&bars->acc_empty[buf], ((n_done >> 1) & 1) ^ 1, bars, status);
+                    // the epilogue warps have read the tile before last out of this accumulator
+                    ok = mbar_wait(&bars->acc_empty[buf], ((n_done >> 1) & 1) ^ 1, cx);
                     if (!ok) break;
                     tc_fence_after();
                 }
                 const uint32_t d_tmem = tmem + buf * kTileN;
                 for (int ks = 0; ks < k_steps; ++ks, ++it) {
                     const int s = it % kStages;
-                    ok = mbar_wait(&bars->full[s], (it / kStages) & 1, bars, status);
+                    ok = mbar_wait(&bars->full[s], (it / kStages) & 1, cx);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t off = (uint64_t)((s * kStageBytes) >> 4);
+                    const uint64_t off = (uint64_t)((s * G::kStageBytes) >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < kTileK / 16; ++kk)   // 16 columns = 32 bytes inside a 128-byte row
-                        mma_ss(d_tmem, a_desc0 + off + 2 * kk, b_desc0 + off + 2 * kk, idesc, (ks | kk) != 0);
-                    tc_commit(&bars->empty[s]);
+                    for (int kk = 0; kk < kTileK / 16; ++kk) { // 16 columns = 32 bytes inside a 128-byte row
+                        if constexpr (PAIR) mma_ss_pair(d_tmem, a_desc0 + off + 2 * kk, b_desc0 + off + 2 * kk, idesc, (ks | kk) != 0);
+                        else mma_ss(d_tmem, a_desc0 + off + 2 * kk, b_desc0 + off + 2 * kk, idesc, (ks | kk) != 0);
+                    }
+                    commit(&bars->empty[s]);
                 }
-                if (ok) tc_commit(&bars->acc_full[buf]);
+                if (ok) commit(&bars->acc_full[buf]);
             }
             if (!ok) {
-                tc_commit(&bars->drain);
+                // gave up: let the MMAs already issued finish (bounded) before TMEM is released
+                commit(&bars->drain);
                 const long long t0 = clock64();
                 while (!mbar_try(&bars->drain, 0) && clock64() - t0 < bars->wait_cycles) { }
             }
@@ -200,125 +354,83 @@ qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUten
         const int quarter = warp & 3;                          // TMEM lanes this warp may touch
         const int row = quarter * 32 + lane;
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-        const int d = a.head_dim, half = d / 2;
-        const int Hq = a.plan.num_heads, Hkv = a.plan.num_kv_heads;
-        const int heads_total = Hq + 2 * Hkv;
-        const bool rotate = a.trig != nullptr;
+        uint32_t lead_empty[2] = {0, 0};                       // CTA 0's acc_empty barriers (pairs)
+        if constexpr (PAIR) {
+            lead_empty[0] = map_to_cta(smem_u32(&bars->acc_empty[0]), 0u);
+            lead_empty[1] = map_to_cta(smem_u32(&bars->acc_empty[1]), 0u);
+        }
         bool ok = true;
         int n_done = 0;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++n_done) {
+        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++n_done) {
             const int m = tile % a.m_tiles, n = tile / a.m_tiles;
             const int buf = n_done & 1;
-            const int t = m * kTileM + row;
-            const bool valid = t < a.plan.total_rows;
-            int64_t pool_off = 0;                              // element offset of (page, slot) in the pools
-            const float2* trig = nullptr;
-            if (valid) {
-                const int r = a.plan.row_req[t];
-                const int p = a.plan.prefix_len[r] + (t - a.plan.cu_chunk[r]);
-                const int page = HAT_IN_RANGE(__ldg(a.plan.block_table + (int64_t)r * a.plan.max_pages +
-                                                    HAT_IN_RANGE(p / kPageSize, a.plan.max_pages, status)),
-                                              a.plan.num_pages, status);
-                pool_off = (int64_t)page * a.cache.stride_page + (int64_t)(p % kPageSize) * a.cache.stride_token;
-                if (rotate) trig = a.trig + (int64_t)t * half;
-            }
-            ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_full[buf], (n_done >> 1) & 1, bars, status));
+            const int t = (PAIR ? m * 2 * kTileM + (int)rank * kTileM : m * kTileM) + row;
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_full[buf], (n_done >> 1) & 1, cx));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t acc = tmem + buf * kTileN + lane_sel;
-
-            for (int hb = 0; hb < kTileN; hb += d) {           // heads of this tile, by their first column in it
-                const int hh = (n * kTileN + hb) / d;
-                if (hh >= heads_total) break;                  // uniform: the feature count does not fill the last tile
-                // where the head's d values go
-                unsigned char* dst;
-                bool rot = rotate;
-                if (hh < Hq) {
-                    dst = static_cast<unsigned char*>(a.q_out) + ((int64_t)t * Hq + hh) * d * 2;
-                } else if (hh < Hq + Hkv) {
-                    dst = static_cast<unsigned char*>(a.k_pool) + (pool_off + (int64_t)(hh - Hq) * a.cache.stride_head) * 2;
-                } else {
-                    dst = static_cast<unsigned char*>(a.v_pool) + (pool_off + (int64_t)(hh - Hq - Hkv) * a.cache.stride_head) * 2;
-                    rot = false;
-                }
-                if (!rot) {
-                    for (int c0 = 0; c0 < d; c0 += 32) {
-                        float v[32];
-                        tmem_ld32(acc + hb + c0, reinterpret_cast<uint32_t*>(v));
-                        tmem_ld_wait();
-                        if (valid) store32<BF16>(dst + c0 * 2, v);
-                    }
-                } else if (a.interleaved) {
-                    // pairs (x[2c], x[2c+1]): 32 columns hold pairs c0/2 .. c0/2 + 15
-                    for (int c0 = 0; c0 < d; c0 += 32) {
-                        float v[32];
-                        tmem_ld32(acc + hb + c0, reinterpret_cast<uint32_t*>(v));
-                        tmem_ld_wait();
-                        if (valid) {
-#pragma unroll
-                            for (int i = 0; i < 16; i += 2) {
-                                const float4 cs = __ldg(reinterpret_cast<const float4*>(trig + c0 / 2 + i));   // two (cos, sin)
-                                const float lo0 = v[2 * i], hi0 = v[2 * i + 1], lo1 = v[2 * i + 2], hi1 = v[2 * i + 3];
-                                v[2 * i] = lo0 * cs.x - hi0 * cs.y;
-                                v[2 * i + 1] = hi0 * cs.x + lo0 * cs.y;
-                                v[2 * i + 2] = lo1 * cs.z - hi1 * cs.w;
-                                v[2 * i + 3] = hi1 * cs.z + lo1 * cs.w;
-                            }
-                            store32<BF16>(dst + c0 * 2, v);
-                        }
-                    }
-                } else {
-                    // pairs (x[c], x[c + d/2]): 32 columns of the low half with their partners of the high half
-                    for (int c0 = 0; c0 < half; c0 += 32) {
-                        float lo[32], hi[32];
-                        tmem_ld32(acc + hb + c0, reinterpret_cast<uint32_t*>(lo));
-                        tmem_ld32(acc + hb + half + c0, reinterpret_cast<uint32_t*>(hi));
-                        tmem_ld_wait();
-                        if (valid) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 2) {
-                                const float4 cs = __ldg(reinterpret_cast<const float4*>(trig + c0 + i));
-                                const float l0 = lo[i], h0 = hi[i], l1 = lo[i + 1], h1 = hi[i + 1];
-                                lo[i] = l0 * cs.x - h0 * cs.y;
-                                hi[i] = h0 * cs.x + l0 * cs.y;
-                                lo[i + 1] = l1 * cs.z - h1 * cs.w;
-                                hi[i + 1] = h1 * cs.z + l1 * cs.w;
-                            }
-                            store32<BF16>(dst + c0 * 2, lo);
-                            store32<BF16>(dst + (half + c0) * 2, hi);
-                        }
-                    }
-                }
-            }
+            epilogue_row<BF16>(a, tmem + buf * kTileN + lane_sel, t, n, cx.status);
             // every value of this accumulator is in registers or stored: hand it back
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->acc_empty[buf]);
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_remote(lead_empty[buf]);
+                else mbar_arrive(&bars->acc_empty[buf]);
+            }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) {
+        // both CTAs are done with each other's barriers, and every MMA has finished, before tensor memory is freed
+        cluster_arrive();
+        cluster_wait();
+    }
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
+        if constexpr (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
     }
+}
+
+template <bool BF16, bool PAIR>
+cudaError_t launch_form(const QkvArgs& a, const CUtensorMap& mx, const CUtensorMap& mw, int num_sms, cudaStream_t stream) {
+    auto kern = qkv_gemm_kernel<BF16, PAIR>;
+    constexpr uint32_t smem = smem_bytes<PAIR>();
+    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), (int)smem);
+    if (e != cudaSuccess) return e;
+    const int tiles = a.m_tiles * a.n_tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    if (PAIR) {
+        cfg.gridDim = dim3((unsigned)(2 * std::min(num_sms / 2, tiles)));
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    } else {
+        cfg.gridDim = dim3((unsigned)std::min(num_sms, tiles));
+    }
+    e = cudaLaunchKernelEx(&cfg, kern, a, mx, mw);
+    count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
 
-size_t qkv_workspace_bytes(const hat_plan* plan) {
-    return (size_t)plan->total_rows * (plan->head_dim / 2) * sizeof(float2);
-}
-
 cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* k_pool, void* v_pool, const void* x,
-                            int hidden, const void* w, void* q_out, float theta, int interleaved, void* workspace,
-                            cudaStream_t stream) {
+                            int hidden, const void* w, void* q_out, float theta, int interleaved, cudaStream_t stream) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     const int d = plan->head_dim, T = plan->total_rows;
     const int64_t features = (int64_t)(plan->num_heads + 2 * plan->num_kv_heads) * d;
+    // pairs of CTAs work on 256 rows at a time; a batch that fits one 128-row tile would leave the second CTA idle
+    const bool pair = T > kTileM;
     CUtensorMap mx, mw;
-    if (!tma_encode_matrix_map(&mx, bf16, x, T, hidden, kTileM) || !tma_encode_matrix_map(&mw, bf16, w, features, hidden, kTileN))
+    if (!tma_encode_matrix_map(&mx, bf16, x, T, hidden, kTileM) ||
+        !tma_encode_matrix_map(&mw, bf16, w, features, hidden, pair ? kTileN / 2 : kTileN))
         return cudaErrorInvalidValue;
     QkvArgs a;
     a.plan = plan->dev;
@@ -326,26 +438,35 @@ cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* 
     a.k_pool = k_pool; a.v_pool = v_pool; a.q_out = q_out;
     a.trig = nullptr;
     a.hidden = hidden; a.head_dim = d; a.interleaved = interleaved;
-    a.m_tiles = (T + kTileM - 1) / kTileM;
+    a.m_tiles = pair ? (T + 2 * kTileM - 1) / (2 * kTileM) : 1;
     a.n_tiles = (int)((features + kTileN - 1) / kTileN);
     a.wait_cycles = plan->wait_cycles;
+    cudaError_t e;
     if (theta > 0.f) {
-        InvFreq fr;
-        for (int c = 0; c < d / 2; ++c) fr.f[c] = std::pow((double)theta, -2.0 * c / d);
-        const int64_t total = (int64_t)T * (d / 2);
-        rope_table_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(plan->dev, d / 2, fr, static_cast<float2*>(workspace));
-        count_launch();
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        a.trig = static_cast<const float2*>(workspace);
+        // the table of cosines and sines depends on the plan's positions and on the base only: every layer of a step
+        // uses the one its first call filled
+        hat_plan* mp = const_cast<hat_plan*>(plan);
+        if (mp->rope_theta != theta) {
+            InvFreq fr;
+            for (int c = 0; c < 64; ++c) fr.f[c] = c < d / 2 ? std::pow((double)theta, -2.0 * c / d) : 0.0;
+            const int64_t total = (int64_t)T * (d / 2);
+            // a call with the previous base may still be reading the table that is about to be replaced (rare: one
+            // model has one base)
+            if (mp->rope_theta > 0.f && (e = cudaDeviceSynchronize()) != cudaSuccess) return e;
+            rope_table_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(plan->dev, d / 2, fr, mp->rope_table);
+            count_launch();
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            if ((e = cudaEventRecord(mp->ev_table, stream)) != cudaSuccess) return e;
+            mp->rope_theta = theta;
+            mp->table_stream = stream;
+        } else if (mp->table_stream != stream) {
+            if ((e = cudaStreamWaitEvent(stream, mp->ev_table, 0)) != cudaSuccess) return e;
+        }
+        a.trig = mp->rope_table;
     }
-    auto kern = bf16 ? qkv_gemm_kernel<true> : qkv_gemm_kernel<false>;
-    cudaError_t e = smem_attr_once(reinterpret_cast<const void*>(kern), (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    const int ctas = std::min(plan->num_sms, a.m_tiles * a.n_tiles);
-    kern<<<dim3((unsigned)ctas), kThreads, kSmemBytes, stream>>>(a, mx, mw);
-    count_launch();
-    return cudaGetLastError();
+    if (pair) e = bf16 ? launch_form<true, true>(a, mx, mw, plan->num_sms, stream) : launch_form<false, true>(a, mx, mw, plan->num_sms, stream);
+    else e = bf16 ? launch_form<true, false>(a, mx, mw, plan->num_sms, stream) : launch_form<false, false>(a, mx, mw, plan->num_sms, stream);
+    return e;
 }
 
 }  // namespace hat

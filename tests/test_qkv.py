@@ -108,29 +108,29 @@ def _run_projection(cuda_device, dtype, d, hq, hkv, hidden, prefix, chunk, theta
     x_dev = runner._dev_u16(xb, cuda_device)
     w_dev = runner._dev_u16(wb, cuda_device)
     g_q = runner._Guarded((T, hq, d), torch.int16, -1, cuda_device)
-    ws_bytes = B.hat_qkv_workspace_bytes(ds.plan)
-    g_ws = runner._Guarded((max(ws_bytes, 256),), torch.uint8, None, cuda_device)
-    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, g_q.view, theta, interleaved, g_ws.view, ws_bytes)
+    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, g_q.view, theta, interleaved)
     torch.cuda.synchronize()
     assert B.hat_last_device_status(ds.plan) == B.HAT_OK
-    assert g_q.intact() and g_ws.intact(), "a canary zone around q_out / workspace was overwritten"
+    assert g_q.intact(), "a canary zone around q_out was overwritten"
     got_q = g_q.view.cpu().numpy().view(np.uint16).reshape(T, hq, d)
     gk, gv = cache.pools_to_host()
     return sc, st, ds, cache, xb, wb, got_q, gk, gv
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("dtype,d,hq,hkv,hidden,theta,interleaved", [
-    ("fp16", 128, 4, 2, 320, 10000.0, False),      # 4 feature tiles, 5 stages of the hidden dimension (the ring wraps)
-    ("bf16", 128, 2, 2, 64, 10000.0, True),        # one stage per tile
-    ("bf16", 64, 6, 3, 128, 10000.0, True),        # four heads per feature tile
-    ("fp16", 64, 3, 1, 192, 500000.0, False),      # 320 features: the second feature tile is partly empty
-    ("fp16", 128, 3, 1, 128, 0.0, False),          # no rotation; 5 heads: the last tile holds one
+@pytest.mark.parametrize("dtype,d,hq,hkv,hidden,theta,interleaved,small", [
+    ("fp16", 128, 4, 2, 448, 10000.0, False, False),   # 4 feature tiles, 7 stages of the hidden dimension (the ring wraps)
+    ("bf16", 128, 2, 2, 64, 10000.0, True, False),     # one stage per tile
+    ("bf16", 64, 6, 3, 128, 10000.0, True, False),     # four heads per feature tile
+    ("fp16", 64, 3, 1, 192, 500000.0, False, False),   # 320 features: the second feature tile is partly empty
+    ("fp16", 128, 3, 1, 128, 0.0, False, False),       # no rotation; 5 heads: the last tile holds one
+    ("bf16", 128, 4, 2, 320, 10000.0, False, True),    # at most 128 rows: the one-CTA form (5 stages, ring of 4)
+    ("fp16", 64, 3, 1, 64, 10000.0, True, True),
 ])
-def test_projection_kernel_rotates_and_appends(cuda_device, dtype, d, hq, hkv, hidden, theta, interleaved):
+def test_projection_kernel_rotates_and_appends(cuda_device, dtype, d, hq, hkv, hidden, theta, interleaved, small):
     """hat_qkv_rope_append against the float64 projection, rotation and append: q rows, the written slots of both
-    pools (and nothing but them), over several row tiles with a ragged last one."""
-    prefix, chunk = [0, 37, 1000, 4090, 8000, 250], [5, 130, 16, 200, 8, 0]
+    pools (and nothing but them).  359 rows (CTA pairs, a ragged second pair of row tiles) or 100 rows (single CTAs)."""
+    prefix, chunk = ([0, 37, 4090], [5, 80, 15]) if small else ([0, 37, 1000, 4090, 8000, 250], [5, 130, 16, 200, 8, 0])
     sc, st, ds, cache, xb, wb, got_q, gk, gv = _run_projection(cuda_device, dtype, d, hq, hkv, hidden, prefix, chunk,
                                                                theta, interleaved)
     pos = R.positions(st)
@@ -189,17 +189,15 @@ def test_projection_kernel_rejects_what_it_cannot_run(cuda_device):
     x = torch.zeros(16 * 96, dtype=torch.int16, device=cuda_device)
     w = torch.zeros(384 * 96, dtype=torch.int16, device=cuda_device)
     q = torch.zeros(16 * 128, dtype=torch.int16, device=cuda_device)
-    ws = torch.zeros(B.hat_qkv_workspace_bytes(ds.plan), dtype=torch.uint8, device=cuda_device)
     L = B.lib()
     import ctypes as C
-    def call(hidden, theta, ws_t, ws_n, xp=x):
-        return L.hat_qkv_rope_append(C.byref(cache.desc), B._h(ds.plan),
-                                     B._ptr(xp), hidden, B._ptr(w), B._ptr(q), C.c_float(theta), 0, B._ptr(ws_t), ws_n, None)
-    assert call(96, 10000.0, ws, ws.numel()) == B.HAT_ERR_UNSUPPORTED            # hidden not a multiple of 64
-    assert call(64, 0.5, ws, ws.numel()) == B.HAT_ERR_INVALID_ARG                # a base in (0, 1]
-    assert call(64, 10000.0, None, 0) == B.HAT_ERR_INVALID_ARG                   # rotation without its table
-    assert call(64, 10000.0, ws, 8) == B.HAT_ERR_WORKSPACE_TOO_SMALL
-    assert call(64, 10000.0, ws, ws.numel(), xp=None) == B.HAT_ERR_INVALID_ARG
-    assert call(64, 10000.0, ws, ws.numel()) == B.HAT_OK
+    def call(hidden, theta, xp=x):
+        return L.hat_qkv_rope_append(C.byref(cache.desc), B._h(ds.plan), B._ptr(xp), hidden, B._ptr(w), B._ptr(q),
+                                     C.c_float(theta), 0, None)
+    assert call(96, 10000.0) == B.HAT_ERR_UNSUPPORTED                            # hidden not a multiple of 64
+    assert call(64, 0.5) == B.HAT_ERR_INVALID_ARG                                # a base in (0, 1]
+    assert call(0, 10000.0) == B.HAT_ERR_INVALID_ARG
+    assert call(64, 10000.0, xp=None) == B.HAT_ERR_INVALID_ARG
+    assert call(64, 10000.0) == B.HAT_OK
     torch.cuda.synchronize()
     ds.close()
