@@ -271,6 +271,58 @@ def quick_config(name, device, stream, peaks, peak_kind, K=20, warmup=3, with_or
     return res
 
 
+def layer_front(sc, cache, ds, device, stream, peaks, peak_kind, K=20, warmup=3, with_oracle=True):
+    """The step in front of the attention module for the first call of the workload (Sec. 2.1: Q = X W_Q, K = X W_K,
+    V = X W_V): the projection kernel with the rotation and the cache write in its epilogue, hidden = heads x head_dim.
+    K timed launches with the L2 flushed in between; a few rows against the float64 oracle."""
+    import torch
+    from paper_2503_18989_b200 import binding as B
+    from paper_2503_18989_b200 import runner
+    st = sc.steps[0]
+    spec = sc.cache
+    hq, hkv, d = int(st.q.shape[1]), spec.num_heads, spec.head_dim
+    hidden, feats, T = hq * d, (hq + 2 * hkv) * d, st.total_rows
+    xb, wb = W.projection_inputs(900, spec.dtype, T, hidden, feats)
+    x_dev, w_dev = runner._dev_u16(xb, device), runner._dev_u16(wb, device)
+    q_out = torch.empty((T, hq, d), dtype=torch.int16, device=device)
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+    launches0 = B.hat_launch_count()
+    for _ in range(warmup):
+        B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q_out, 10000.0, False, stream)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in evs:
+        flush_buf.zero_()
+        a.record()
+        B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q_out, 10000.0, False, stream)
+        b.record()
+    torch.cuda.synchronize(device)
+    ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+    flops = 2.0 * T * hidden * feats
+    tensor_peak, source = pick_tensor_peak(peaks, peak_kind, K * ms * 1e-3, [])
+    e = 2
+    res = {"op": "qkv projection + rotation + cache write (hat_qkv_rope_append)", "rows": T, "hidden": hidden,
+           "features": feats, "dtype": spec.dtype, "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+           "bound": "tensor", "peak": tensor_peak, "peak_source": source,
+           "frac": flops / (ms * 1e-3) / 1e12 / tensor_peak,
+           "frac_nominal": flops / (ms * 1e-3) / 1e12 / NOMINAL["tensor_tflops"],
+           "algorithmic_bytes": (T * hidden + feats * hidden + T * feats) * e,
+           "launches": (B.hat_launch_count() - launches0) // (warmup + K),
+           "device_status_ok": B.hat_last_device_status(ds.plan, stream) == B.HAT_OK}
+    if with_oracle:
+        from oracle import hat_qkv_oracle as QO
+        from oracle import hat_rope_oracle as RO
+        rows = np.unique(np.random.default_rng(2).integers(0, T, size=16))
+        pos = RO.positions(st)
+        want_q, _, _ = QO.qkv_rope(xb[rows], wb, pos[rows], spec.dtype, hq, hkv, d)
+        got_q = q_out[torch.from_numpy(rows).to(device)].cpu().numpy().view(np.uint16)
+        gw, ww = W.bits_to_f64(got_q, spec.dtype), W.bits_to_f64(want_q, spec.dtype)
+        res["oracle_sample"] = {"rows": int(len(rows)), "same_bits_share": float(np.mean(got_q == want_q)),
+                                "max_abs_q": float(np.abs(gw - ww).max())}
+    del x_dev, w_dev, q_out, flush_buf
+    torch.cuda.empty_cache()
+    return res
+
+
 def lookup_traffic(kernel: str, workload: str):
     """DRAM bytes per launch from the committed ncu capture of this kernel on this workload, or None when
     there is none or the kernel source has changed since (profiles/traffic.json records a source hash)."""
@@ -624,6 +676,11 @@ def main():
         if args.all_configs and world == 1:
             # the other named workloads, briefly, so that all five are in this run's record (parity cases, not the
             # headline: the line's value and roofline stay those of config.workload)
+            try:
+                line["layer_front"] = layer_front(sc, cache, steps[0], device, stream, peaks, peak_kind,
+                                                  with_oracle=not args.no_cpu_baseline)
+            except Exception as exc:
+                line["layer_front"] = {"error": str(exc)}
             for ds in steps:
                 ds.close()
             del steps, cache, flush_buf, host

@@ -201,3 +201,57 @@ def test_projection_kernel_rejects_what_it_cannot_run(cuda_device):
     assert call(64, 10000.0) == B.HAT_OK
     torch.cuda.synchronize()
     ds.close()
+
+
+@pytest.mark.gpu
+def test_projection_at_the_13b_mixed_batch_size_on_sampled_rows(cuda_device):
+    """The projection of the 13B-shaped mixed batch (4224 rows, hidden 5120, 40 + 40 + 40 heads of 128, bf16) in the
+    launch configuration the benchmark times: sampled rows (first and last row of prefill and verify requests, random
+    others) against the float64 oracle, q rows and the K / V slots read back through the block table."""
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    sc = W.mixed_13b()
+    st = sc.steps[0]
+    spec = sc.cache
+    dtype, d, hkv = spec.dtype, spec.head_dim, spec.num_heads
+    hq = int(st.q.shape[1])
+    hidden = hq * d
+    T = st.total_rows
+    feats = (hq + 2 * hkv) * d
+    xb, wb = W.projection_inputs(900, dtype, T, hidden, feats)
+    cache = runner.DeviceCache(spec, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    x_dev, w_dev = runner._dev_u16(xb, cuda_device), runner._dev_u16(wb, cuda_device)
+    g_q = runner._Guarded((T, hq, d), torch.int16, -1, cuda_device)
+    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, g_q.view, 10000.0, False)
+    torch.cuda.synchronize()
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    assert g_q.intact()
+
+    rng = np.random.default_rng(4)
+    pos = R.positions(st)
+    rows = set(int(t) for t in rng.integers(0, T, size=24))
+    for r in list(range(0, st.num_requests, 7)) + [st.num_requests - 1]:
+        if st.chunk_len[r] > 0:
+            rows.update((int(st.cu_chunk[r]), int(st.cu_chunk[r + 1]) - 1))
+    rows = np.asarray(sorted(rows))
+    req = np.searchsorted(st.cu_chunk, rows, side="right") - 1
+    want_q, want_k, want_v = QO.qkv_rope(xb[rows], wb, pos[rows], dtype, hq, hkv, d)
+    got_q = g_q.view[torch.from_numpy(rows).to(cuda_device)].cpu().numpy().view(np.uint16)
+    _assert_projected(got_q, want_q, dtype, "sampled q rows", 0.97)
+    # element offsets of the sampled rows' slots: [row][head][d]
+    page = st.block_table[req, pos[rows] // spec.page_size].astype(np.int64)
+    base = page * spec.stride_page + (pos[rows] % spec.page_size) * spec.stride_token
+    offs = base[:, None, None] + (np.arange(hkv, dtype=np.int64) * spec.stride_head)[None, :, None] + np.arange(d)[None, None, :]
+    idx = torch.from_numpy(offs.reshape(-1)).to(cuda_device)
+    got_k = cache.k.view(-1)[idx].cpu().numpy().view(np.uint16).reshape(len(rows), hkv, d)
+    got_v = cache.v.view(-1)[idx].cpu().numpy().view(np.uint16).reshape(len(rows), hkv, d)
+    _assert_projected(got_k, want_k, dtype, "sampled K slots", 0.97)
+    _assert_projected(got_v, want_v, dtype, "sampled V slots", 0.97)
+    # the slot behind a request's last row belongs to nobody yet and keeps its content
+    for r in (0, st.num_requests - 1):
+        p_next = int(st.prefix_len[r] + st.chunk_len[r])
+        if p_next // spec.page_size < st.max_pages and st.block_table[r, p_next // spec.page_size] >= 0:
+            o = int(st.block_table[r, p_next // spec.page_size]) * spec.stride_page + (p_next % spec.page_size) * spec.stride_token
+            assert np.array_equal(cache.k.view(-1)[o:o + d].cpu().numpy().view(np.uint16), sc.k_pool[o:o + d])
+    ds.close()
