@@ -439,6 +439,8 @@ def main():
                     help="after the main measurement, time the other named workloads briefly (default: on for the default "
                          "workload on one GPU)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
+    ap.add_argument("--layer-front", dest="layer_front", action="store_true", default=None,
+                    help="also time the projection kernel in front of the attention step (default: with --all-configs)")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
     args = ap.parse_args()
     if args.all_configs is None:
@@ -673,14 +675,15 @@ def main():
             rate, cores, sample, _, _ = time_oracle(sc, args.cpu_budget)
             line["cpu_baseline"] = {"value": rate / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                     "sample": sample}
-        if args.all_configs and world == 1:
-            # the other named workloads, briefly, so that all five are in this run's record (parity cases, not the
-            # headline: the line's value and roofline stay those of config.workload)
+        if (args.layer_front or (args.layer_front is None and args.all_configs)) and world == 1:
             try:
                 line["layer_front"] = layer_front(sc, cache, steps[0], device, stream, peaks, peak_kind,
                                                   with_oracle=not args.no_cpu_baseline)
             except Exception as exc:
                 line["layer_front"] = {"error": str(exc)}
+        if args.all_configs and world == 1:
+            # the other named workloads, briefly, so that all five are in this run's record (parity cases, not the
+            # headline: the line's value and roofline stay those of config.workload)
             for ds in steps:
                 ds.close()
             del steps, cache, flush_buf, host
