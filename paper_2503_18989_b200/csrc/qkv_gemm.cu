@@ -4,19 +4,19 @@
 //
 //   y[t][f] = sum_j x[t][j] w[f][j]        x [T][hidden], w [(Hq + 2 Hkv) d][hidden] (one row per output feature),
 //                                          features ordered q heads | k heads | v heads
-// Persistent kernel, output tiles of 256 features (two heads of 128 or four of 64), drawn in a fixed order with the row
-// tile running fastest: the CTAs of one round share a strip of w, which then crosses HBM once, and x (much smaller)
-// stays in L2.  Two forms:
-//   PAIR   clusters of two CTAs, tcgen05.mma.cta_group::2 with M = 256: each CTA stages its own 128 rows of x and
-//          HALF of the 256 rows of w (32 KiB per 64 columns of the hidden dimension and CTA, six stages).  What bounds
-//          this GEMM on 148 SMs is the path from L2 into shared memory, and a pair moves 2/3 of the bytes per flop that
-//          two single CTAs do
-//   single one CTA per tile of 128 rows (48 KiB per stage, four stages): batches of at most 128 rows, which would leave
-//          half of a pair idle
+// Persistent kernel, output tiles of whole heads, drawn in a fixed order with the row tile running fastest: the CTAs of
+// one round share a strip of w, which then crosses HBM once, and x (much smaller) stays in L2.  Two forms:
+//   PAIR   clusters of two CTAs, tcgen05.mma.cta_group::2 with M = 256, tiles of 256 features (two heads of 128 or four
+//          of 64): each CTA stages its own 128 rows of x and HALF of the 256 rows of w (32 KiB per 64 columns of the
+//          hidden dimension and CTA, six stages).  What bounds this GEMM on 148 SMs is the path from L2 into shared
+//          memory, and a pair moves 2/3 of the bytes per flop that two single CTAs with 128 x 256 tiles do
+//   single batches of at most 128 rows (draft verification), which would leave half of a pair idle and are bound by
+//          reading w once from HBM: one CTA per tile of 128 rows x 128 features, so that twice as many SMs pull on w
+//          (120 tiles at the 13B shape, where 256-feature tiles gave 60 and 57 us against 40)
 // Roles (per CTA):
 //   warp 0      TMA producer: per 64 columns of the hidden dimension one box of x and one of w, 128-byte swizzle
 //   warp 1      CTA 0 of a pair (or the single CTA): one thread issues tcgen05.mma (four per stage) into one of two
-//               256-column accumulators in TMEM; tcgen05.commit frees the stage (in both CTAs) and, after the last
+//               accumulators (256 or 128 columns) in TMEM; tcgen05.commit frees the stage (in both CTAs) and, after the last
 //               stage of a tile, hands the accumulator to the epilogue warps.  CTA 1: one thread forwards "my half of
 //               this stage has landed" to CTA 0's barrier.  The warp owns the TMEM allocation
 //   warps 2-5   epilogue, thread = output row = TMEM lane: reads the accumulator 32 columns at a time, rotates q and k
@@ -32,6 +32,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 
 #include "hat_internal.h"
 #include "tma_desc.h"
@@ -41,14 +42,15 @@ namespace hat {
 namespace {
 using namespace tc5;
 
-constexpr int kTileM = 128, kTileN = 256, kTileK = 64;
+constexpr int kTileM = 128, kTileK = 64;
 constexpr uint32_t kABytes = kTileM * kTileK * 2;        // 16 KiB: 128 rows of x
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 6;
 
 template <bool PAIR> struct Geo {
-    static constexpr int kStages = PAIR ? 6 : 4;
-    static constexpr int kBRows = PAIR ? kTileN / 2 : kTileN;            // rows of w one CTA stages
+    static constexpr int kStages = 6;
+    static constexpr int kTileN = PAIR ? 256 : 128;                      // features per output tile
+    static constexpr int kBRows = 128;                                   // rows of w one CTA stages (half a tile for pairs)
     static constexpr uint32_t kBBytes = kBRows * kTileK * 2;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
 };
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(256) rope_table_kernel(DevicePlan plan, int ha
 }
 
 // One output row of one tile: the thread's TMEM lane of the accumulator at `acc`, packed row t, feature tile n.
-template <bool BF16>
+template <bool BF16, int kTileN>
 __device__ __forceinline__ void epilogue_row(const QkvArgs& a, uint32_t acc, int t, int n, int32_t* status) {
     const int d = a.head_dim, half = d / 2;
     const int Hq = a.plan.num_heads, Hkv = a.plan.num_kv_heads;
@@ -215,6 +217,7 @@ qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUten
                 const __grid_constant__ CUtensorMap map_w) {
     using G = Geo<PAIR>;
     constexpr int kStages = G::kStages;
+    constexpr int kTileN = G::kTileN;
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the swizzle pattern; both CTAs of a pair get the same offsets (one descriptor serves both)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -368,7 +371,7 @@ qkv_gemm_kernel(const __grid_constant__ QkvArgs a, const __grid_constant__ CUten
             ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_full[buf], (n_done >> 1) & 1, cx));
             if (!ok) break;
             tc_fence_after();
-            epilogue_row<BF16>(a, tmem + buf * kTileN + lane_sel, t, n, cx.status);
+            epilogue_row<BF16, kTileN>(a, tmem + buf * kTileN + lane_sel, t, n, cx.status);
             // every value of this accumulator is in registers or stored: hand it back
             tc_fence_before();
             __syncwarp();
@@ -427,10 +430,13 @@ cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* 
     const int d = plan->head_dim, T = plan->total_rows;
     const int64_t features = (int64_t)(plan->num_heads + 2 * plan->num_kv_heads) * d;
     // pairs of CTAs work on 256 rows at a time; a batch that fits one 128-row tile would leave the second CTA idle
-    const bool pair = T > kTileM;
+    // (HAT_QKV_PAIR_ROWS overrides the row count above which pairs are used, for tuning)
+    int pair_rows = kTileM;
+    if (const char* v = std::getenv("HAT_QKV_PAIR_ROWS")) pair_rows = std::max(0, std::atoi(v));
+    const bool pair = T > pair_rows;
     CUtensorMap mx, mw;
     if (!tma_encode_matrix_map(&mx, bf16, x, T, hidden, kTileM) ||
-        !tma_encode_matrix_map(&mw, bf16, w, features, hidden, pair ? kTileN / 2 : kTileN))
+        !tma_encode_matrix_map(&mw, bf16, w, features, hidden, 128))
         return cudaErrorInvalidValue;
     QkvArgs a;
     a.plan = plan->dev;
@@ -438,8 +444,9 @@ cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* 
     a.k_pool = k_pool; a.v_pool = v_pool; a.q_out = q_out;
     a.trig = nullptr;
     a.hidden = hidden; a.head_dim = d; a.interleaved = interleaved;
-    a.m_tiles = pair ? (T + 2 * kTileM - 1) / (2 * kTileM) : 1;
-    a.n_tiles = (int)((features + kTileN - 1) / kTileN);
+    a.m_tiles = pair ? (T + 2 * kTileM - 1) / (2 * kTileM) : (T + kTileM - 1) / kTileM;
+    const int tile_n = pair ? Geo<true>::kTileN : Geo<false>::kTileN;
+    a.n_tiles = (int)((features + tile_n - 1) / tile_n);
     a.wait_cycles = plan->wait_cycles;
     cudaError_t e;
     if (theta > 0.f) {
