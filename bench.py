@@ -308,6 +308,22 @@ def layer_front(sc, cache, ds, device, stream, peaks, peak_kind, K=20, warmup=3,
            "algorithmic_bytes": (T * hidden + feats * hidden + T * feats) * e,
            "launches": (B.hat_launch_count() - launches0) // (warmup + K),
            "device_status_ok": B.hat_last_device_status(ds.plan, stream) == B.HAT_OK}
+    # the attention step on the projection's own q rows and on the cache it wrote: no append kernel, no k_new / v_new
+    # read (the projection's cache write stands in for it), timed as projection + attention back to back
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(K)]
+    for a, m, b in evs:
+        flush_buf.zero_()
+        a.record()
+        B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q_out, 10000.0, False, stream)
+        m.record()
+        B.hat_chunk_attention(cache.desc, ds.plan, q_out, None, None, ds.out, ds.lse, 0.0, ds.workspace,
+                              ds.workspace_bytes, stream)
+        b.record()
+    torch.cuda.synchronize(device)
+    res["then_attention_without_append_ms"] = float(np.median([m.elapsed_time(b) for a, m, b in evs]))
+    res["projection_and_attention_ms"] = float(np.median([a.elapsed_time(b) for a, m, b in evs]))
+    res["device_status_ok"] = res["device_status_ok"] and B.hat_last_device_status(ds.plan, stream) == B.HAT_OK
     if with_oracle:
         from oracle import hat_qkv_oracle as QO
         from oracle import hat_rope_oracle as RO
