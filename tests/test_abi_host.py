@@ -103,6 +103,9 @@ def test_host_only_plan_cannot_launch(hat_lib):
     c = _cache()
     p = _plan(c, [10], [4], [[0]])
     assert hat_lib.hat_kv_append(C.byref(c), p.handle, None, None, None) == B.HAT_ERR_INVALID_ARG
+    assert hat_lib.hat_qkv_rope_append(C.byref(c), p.handle, None, 64, None, None, C.c_float(10000.0), 0,
+                                       None) == B.HAT_ERR_INVALID_ARG
+    assert hat_lib.hat_qkv_rope_append(None, None, None, 64, None, None, C.c_float(10000.0), 0, None) == B.HAT_ERR_INVALID_ARG
 
 
 def _info(sc, step=0, **env):

@@ -255,3 +255,38 @@ def test_projection_at_the_13b_mixed_batch_size_on_sampled_rows(cuda_device):
             o = int(st.block_table[r, p_next // spec.page_size]) * spec.stride_page + (p_next % spec.page_size) * spec.stride_token
             assert np.array_equal(cache.k.view(-1)[o:o + d].cpu().numpy().view(np.uint16), sc.k_pool[o:o + d])
     ds.close()
+
+
+@pytest.mark.gpu
+def test_projection_on_two_streams_and_with_two_bases(cuda_device):
+    """The table of cosines and sines belongs to the plan: a call on another stream than the one that filled it is
+    ordered behind the fill, and a call with another base refills it.  Same results as single-stream calls."""
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    dtype, d, hq, hkv, hidden = "fp16", 128, 2, 1, 128
+    prefix, chunk = [0, 500, 4000], [140, 3, 60]
+    rng = np.random.Generator(np.random.PCG64(21))
+    table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=2)
+    st = W._make_step(321, dtype, hkv, d, prefix, chunk, table, q_heads=hq)
+    sc = W._scenario("qkv", dtype, hkv, d, "paged", num_pages, [st], 321)
+    T = st.total_rows
+    xb, wb = W.projection_inputs(55, dtype, T, hidden, (hq + 2 * hkv) * d)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    x_dev, w_dev = runner._dev_u16(xb, cuda_device), runner._dev_u16(wb, cuda_device)
+    s1, s2 = torch.cuda.Stream(cuda_device), torch.cuda.Stream(cuda_device)
+    torch.cuda.synchronize()
+    pos = R.positions(st)
+    outs = {}
+    for theta, stream in ((10000.0, s1), (10000.0, s2), (500000.0, s2), (500000.0, s1)):
+        q = torch.full((T, hq, d), -1, dtype=torch.int16, device=cuda_device)
+        B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q, theta, False, stream.cuda_stream)
+        outs.setdefault(theta, []).append(q)
+    torch.cuda.synchronize()
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    for theta, qs in outs.items():
+        want_q, _, _ = QO.qkv_rope(xb, wb, pos, dtype, hq, hkv, d, theta)
+        a, b = (t.cpu().numpy().view(np.uint16) for t in qs)
+        assert np.array_equal(a, b), "the same call on another stream gives other bits"
+        _assert_projected(a, want_q, dtype, f"q rows, base {theta}", 0.97)
+    ds.close()
