@@ -268,6 +268,20 @@ def test_host_buffer_entry_point(cuda_device):
     assert_parity(lse.numpy(), want[0][1], "host entry lse")
     gk, gv = cache.pools_to_host()
     assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+    # two steps in flight, as the benchmark's end-to-end leg runs them: alternate streams, each with its own staging
+    # and result buffers; the copies of one overlap the other's kernels, the plan keeps the kernels in order
+    streams = [torch.cuda.Stream(cuda_device), torch.cuda.Stream(cuda_device)]
+    outs = [(torch.full((T, H, d), float("nan"), dtype=torch.float32).pin_memory(),
+             torch.full((T, H), float("nan"), dtype=torch.float32).pin_memory(),
+             torch.empty(nbytes, dtype=torch.uint8, device=cuda_device)) for _ in streams]
+    for i in range(6):
+        o, l, stg = outs[i % 2]
+        B.hat_chunk_attention_host(cache.desc, ds.plan, q, k, v, o, l, 0.0, stg, nbytes, ds.workspace,
+                                   ds.workspace_bytes, streams[i % 2].cuda_stream)
+    torch.cuda.synchronize()
+    for o, l, _ in outs:
+        assert_parity(o.numpy(), want[0][0], "host entry, two in flight, out")
+        assert_parity(l.numpy(), want[0][1], "host entry, two in flight, lse")
 
 
 def test_bounded_wait_gives_up_and_the_context_stays_usable(cuda_device):
