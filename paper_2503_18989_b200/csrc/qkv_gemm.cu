@@ -12,7 +12,7 @@
 //          memory, and a pair moves 2/3 of the bytes per flop that two single CTAs with 128 x 256 tiles do
 //   single batches of at most 128 rows (draft verification), which would leave half of a pair idle and are bound by
 //          reading w once from HBM: one CTA per tile of 128 rows x 128 features, so that twice as many SMs pull on w
-//          (120 tiles at the 13B shape, where 256-feature tiles gave 60 and 57 us against 40)
+//          (120 tiles at the 13B shape: 47 us, where 256-feature tiles gave 60 tiles and 57 us)
 // Roles (per CTA):
 //   warp 0      TMA producer: per 64 columns of the hidden dimension one box of x and one of w, 128-byte swizzle
 //   warp 1      CTA 0 of a pair (or the single CTA): one thread issues tcgen05.mma (four per stage) into one of two
