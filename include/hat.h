@@ -327,15 +327,17 @@ int hat_plan_wait_verify(const hat_plan* plan);
 int hat_last_device_status(const hat_plan* plan, void* stream, int* out);
 
 /*
- * Failure detection of the tile kernel.  Every wait inside it (on a TMA
- * transfer, on the tensor pipe, on another warp) is bounded by `cycles` SM
- * clock cycles (0 selects the default of 2e9, about a second); a wait that
- * runs out sets the status word above, tells the other warps of its CTA to
- * stop, and the CTA releases its tensor memory and exits.
+ * Failure detection of the tcgen05 kernels (tile attention, projection).
+ * Every wait inside them (on a TMA transfer, on the tensor pipe, on another
+ * warp or the other CTA of a pair) is bounded by `cycles` SM clock cycles (0
+ * selects the default of 2e9, about a second); a wait that runs out sets the
+ * status word above, tells the other warps of its CTA (and the other CTA of
+ * its pair) to stop, and the CTA releases its tensor memory and exits.
  * withhold_next_call != 0 is a self test of that path: in the next
- * hat_chunk_attention call on this plan every tile-kernel CTA skips one of
- * its own transfers, so that a wait does run out within the bound; that call's
- * out/lse are undefined.  Nothing faults or hangs.
+ * hat_chunk_attention or hat_qkv_rope_append call on this plan, whichever
+ * comes first, every CTA that loads skips one of its own transfers, so that
+ * a wait does run out within the bound; that call's results are undefined.
+ * Nothing faults or hangs.
  */
 int hat_plan_set_wait_limit(hat_plan* plan, long long cycles, int withhold_next_call);
 

@@ -290,3 +290,37 @@ def test_projection_on_two_streams_and_with_two_bases(cuda_device):
         assert np.array_equal(a, b), "the same call on another stream gives other bits"
         _assert_projected(a, want_q, dtype, f"q rows, base {theta}", 0.97)
     ds.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows", [300, 100])
+def test_projection_kernel_gives_up_a_wait_and_the_context_stays_usable(cuda_device, rows):
+    """Failure detection without a fault: the producer of CTA 0 (of every pair; 300 rows run on pairs, 100 on single
+    CTAs) withholds its first transfer, the waits on it run out after the shortened bound, both CTAs of a pair wind
+    down, the status word reports it, reading clears it, and the next call is correct."""
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    dtype, d, hq, hkv, hidden = "fp16", 128, 2, 1, 512
+    prefix, chunk = [40, 900], [rows - 20, 20]
+    rng = np.random.Generator(np.random.PCG64(31))
+    table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=2)
+    st = W._make_step(77, dtype, hkv, d, prefix, chunk, table, q_heads=hq)
+    sc = W._scenario("qkv", dtype, hkv, d, "paged", num_pages, [st], 77)
+    T = st.total_rows
+    xb, wb = W.projection_inputs(66, dtype, T, hidden, (hq + 2 * hkv) * d)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    x_dev, w_dev = runner._dev_u16(xb, cuda_device), runner._dev_u16(wb, cuda_device)
+    q = torch.full((T, hq, d), -1, dtype=torch.int16, device=cuda_device)
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    B.hat_plan_set_wait_limit(ds.plan, 20_000_000, withhold_next_call=True)      # about 10 ms
+    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q, 10000.0, False)
+    assert B.hat_last_device_status(ds.plan) == B.HAT_ERR_DEVICE_TIMEOUT
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK                          # reading cleared it
+    B.hat_plan_set_wait_limit(ds.plan, 0, withhold_next_call=False)
+    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q, 10000.0, False)
+    torch.cuda.synchronize()
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    want_q, _, _ = QO.qkv_rope(xb, wb, R.positions(st), dtype, hq, hkv, d)
+    _assert_projected(q.cpu().numpy().view(np.uint16), want_q, dtype, "q rows after the self test", 0.97)
+    ds.close()
