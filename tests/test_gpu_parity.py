@@ -284,15 +284,18 @@ def test_host_buffer_entry_point(cuda_device):
         assert_parity(l.numpy(), want[0][1], "host entry, two in flight, lse")
 
 
-def test_bounded_wait_gives_up_and_the_context_stays_usable(cuda_device):
+@pytest.mark.parametrize("kernel,code", [("tc5", 1), ("pair", 3)])
+def test_bounded_wait_gives_up_and_the_context_stays_usable(cuda_device, kernel, code, monkeypatch):
     """Failure detection without a fault: the tile kernel's producer withholds one transfer, the waiting
-    warps give up after the (shortened) bound, the status word reports it, and the next call is correct."""
+    warps give up after the (shortened) bound (in the CTA-pair kernel both CTAs of every pair), the status word
+    reports it, and the next call is correct."""
     from paper_2503_18989_b200 import binding as B, runner
+    monkeypatch.setenv("HAT_PREFILL_KERNEL", kernel)
     sc = _manual("fp16", 2, 128, [300], [200], 21)
     st = sc.steps[0]
     cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
     ds = runner.DeviceStep(cache, st)
-    assert ds.info["prefill_kernel"] in (1, 3)
+    assert ds.info["prefill_kernel"] == code
     assert B.hat_last_device_status(ds.plan) == B.HAT_OK
     B.hat_plan_set_wait_limit(ds.plan, 20_000_000, withhold_next_call=True)      # about 10 ms
     ds.attend(fused_append=True)
