@@ -28,15 +28,19 @@
 //               commit of P V(g).  Commits are multicast to the barriers of both CTAs.
 //               CTA 1: one thread forwards "my half has landed" of every Q and K load to CTA 0's barriers (the V halves
 //               are checked by the softmax warpgroups before they hand P over).  Both CTAs: owns the TMEM allocation
-//   warps 2-5   softmax warpgroup 0: the tiles with even g          (thread = query row = TMEM lane)
-//   warps 6-9   softmax warpgroup 1: the tiles with odd g
+//   warps 2-5   softmax warpgroup 0   (thread = query row = TMEM lane; the two warpgroups share the CTA's 128 rows)
+//   warps 6-9   softmax warpgroup 1
 //
-// Both warpgroups of a CTA feed the same accumulator, so they share ONE reference maximum per row.  It only moves when
-// a tile's row maximum exceeds it by more than 2^8 (then O is rescaled in TMEM by the warpgroup that moved it, after
-// the previous P V has finished and before its own is issued).  The reference passes from tile g to tile g+1 through
-// shared memory as soon as tile g's row maximum is known, i.e. before its exponentials: the only serial link between
-// consecutive tiles.  Each warpgroup keeps its own row sums; they are combined when the unit ends, and each warpgroup
-// stores one half of the output columns.
+// Both warpgroups of a CTA feed the same accumulator, so a row has ONE reference maximum.  It only moves when a tile's
+// row maximum exceeds it by more than 2^8 (then O is rescaled in TMEM, after the previous P V has finished and before
+// the tile's own is issued).  How a tile is shared depends on the type (measured, see the softmax role below):
+//   fp16   the warpgroups take alternate tiles (even / odd g).  The reference passes from tile g to tile g+1 through
+//          shared memory as soon as tile g's row maximum is known, i.e. before its exponentials: the only serial link
+//          between consecutive tiles.  Each warpgroup keeps its own row sums; they are combined when the unit ends.
+//   bf16   both warpgroups take every tile, 64 keys each: a row has two threads (the same lane of the two warps that
+//          share a lane quarter).  They exchange the maxima of their halves through shared memory every tile and take
+//          the same decisions from them; each keeps the row sum of its keys and rescales its half of O's columns.
+// Either way each warpgroup stores one half of the output columns.
 //
 // Every wait is bounded; a wait that gives up sets the plan's status word and the abort flags of both CTAs, which every
 // other wait observes; both CTAs then still meet at the cluster barrier, free their TMEM and exit normally.
@@ -79,19 +83,22 @@ struct __align__(8) Barriers {
     uint64_t v_full[kStagesV];                              // own loads only: the tile's warpgroup checks it before it arrives on p_ready
     uint64_t k_empty[kStagesK], v_empty[kStagesV];          // pair (a commit costs the issuing thread nothing; a poll does)
     uint64_t s_full[kSBuf], pv_done[kSBuf];                 // pair
-    uint64_t p_ready[kSBuf];                                // CTA 0: the four warps of the tile's warpgroup in each CTA
+    uint64_t p_ready[kSBuf];                                // CTA 0: the softmax warps that work on the tile, of both CTAs
     uint64_t o_free;                                        // CTA 0: all sixteen softmax warps hold their part of O in registers
     uint64_t unit_full[kUnitSlots];                         // own queue, filled by CTA 0's producer
     uint64_t unit_empty[kUnitSlots];                        // CTA 0: every reader of the queue in both CTAs
-    uint64_t m_ready[2][4];                                 // own: warpgroup w, lane quarter q published its tile's reference maximum
-    uint64_t fin_ready[2][4];                               // own: the same for the row-sum hand-over at the end of a unit
+    uint64_t pair_bar[4];                                   // bf16, own: the two warps that share lane quarter q (one of each warpgroup) meet here
+    uint64_t m_ready[2][4];                                 // fp16, own: warpgroup w, lane quarter q published its tile's reference maximum
+    uint64_t fin_ready[2][4];                               // fp16, own: the same for the row-sum hand-over at the end of a unit
     uint64_t drain, drain2;
     long long wait_cycles;                                  // bound of every wait below
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile int unit_slot[kUnitSlots];                     // unit index, or -1 when the work has run out
-    float mref[kRows];                                      // per row: the reference maximum the latest tile left behind
-    float lsum[2][kRows];                                   // [unit parity][row]: row-sum hand-over at the end of a unit
+    float mx_x[2][2][kRows];                                // bf16, [tile parity][warpgroup][row]: maximum over the warpgroup's half of the tile's keys
+    float lsum2[2][2][kRows];                               // bf16, [unit parity][warpgroup][row]: row sum over the warpgroup's keys of the unit
+    float mref[kRows];                                      // fp16, per row: the reference maximum the latest tile left behind
+    float lsum[2][kRows];                                   // fp16, [unit parity][row]: row-sum hand-over at the end of a unit
 };
 constexpr uint32_t kSmemBytes = 1024 /*alignment slack*/ + kTileBytes * 2 + kHalfBytes * (kStagesK + kStagesV) + sizeof(Barriers);
 static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
@@ -190,7 +197,7 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
         for (int s = 0; s < kStagesV; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int s = 0; s < kSBuf; ++s) {
             mbar_init(&bars->s_full[s], 1);
-            mbar_init(&bars->p_ready[s], 8);                     // one arrival per warp of the tile's warpgroup, both CTAs
+            mbar_init(&bars->p_ready[s], BF16 ? 16 : 8);          // one arrival per softmax warp that works on the tile, both CTAs
             mbar_init(&bars->pv_done[s], 1);
         }
         mbar_init(&bars->o_free, 16);
@@ -198,6 +205,7 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
             mbar_init(&bars->unit_full[s], 1);
             mbar_init(&bars->unit_empty[s], kQueueReaders0 + kQueueReaders1);
         }
+        for (int q = 0; q < 4; ++q) mbar_init(&bars->pair_bar[q], 2);
         for (int w = 0; w < 2; ++w)
             for (int q = 0; q < 4; ++q) { mbar_init(&bars->m_ready[w][q], 1); mbar_init(&bars->fin_ready[w][q], 1); }
         mbar_init(&bars->drain, 1);
@@ -540,228 +548,449 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax / correction / output
-        const int w = (warp - 2) >> 2;                      // warpgroup: takes the tiles with g % 2 == w
-        const int quarter = warp & 3;                       // TMEM lanes this warp may touch
-        const int t = quarter * 32 + lane;                  // query row inside this CTA's tile = TMEM lane
-        const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-        const uint32_t tm_o = tmem + kColO + lane_sel;
-        const int wg_tid = (int)threadIdx.x - 64 - w * 128;
-        const float sc = a.scale_log2;
-        const bool wide_stores = ((reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.part_out)) & 31) == 0;
-        const uint32_t lead_o_free = lead(&bars->o_free), lead_p_ready = lead(&bars->p_ready[0]);
-        int g0 = 0;                                         // global index of the unit's first tile
-        bool ok = true;
-        PH_DECL(16);
-        PH_T0(tw0);
-        for (int un = 0; ok; ++un) {
-            const int unit = read_unit(un, true);
-            PH_ADD(0, tw0);
-            if (unit == -2) { ok = false; break; }
-            if (unit < 0) break;
-            const Unit u = decode_unit(a, items, unit);
-            const int i_row = u.row0 + (int)rank * kRows + t;   // row inside the chunk
-            const int last_key = min(u.P + i_row, u.kv_end - 1);
-            float m_mine = -INFINITY, l = 0.f;               // reference this warpgroup's row sum is expressed in; the sum
-            float m_other = -INFINITY;                       // reference the other warpgroup's latest tile of this unit left
-            for (int j = (g0 & 1) == w ? 0 : 1; j < u.n; j += 2) {
-                const int g = g0 + j, b = g % kSBuf;
-                const int kb = u.kv_begin + j * kKeys;
-                const uint32_t tm_s = tmem + b * 128 + lane_sel;
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[b], (g / kSBuf) & 1, cx));
-                if (!ok) break;
-                PH_ADD(1, tw0);
-                tc_fence_after();
-                float s[kKeys];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
-                tmem_ld_wait();
-
-                // raw maximum (the scale is positive, so it commutes with max); four independent chains
-                const int lim = last_key - kb;              // keys 0..lim of this tile are visible to this row
-                if (lim < kKeys - 1) {
-#pragma unroll
-                    for (int k = 0; k < kKeys; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
-                }
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                for (int k = 0; k < kKeys; k += 8) {
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], fmaxf(s[k + 2 * v], s[k + 2 * v + 1]));
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
-                PH_ADD(2, tw0);
-                // the reference the previous tile (the other warpgroup's) left behind
-                float m_prev = -INFINITY;
-                if (j > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->m_ready[w ^ 1][quarter], ((g - 1) >> 1) & 1, cx));
-                    if (!ok) break;
-                    m_prev = bars->mref[t];
-                }
-                PH_ADD(3, tw0);
-                // move it only when this tile's maximum exceeds it by more than the threshold
-                const float m_new = (mx > m_prev + kRescaleThreshold) ? mx : m_prev;
-                const bool rescale = (m_new != m_prev) && (m_prev != -INFINITY);
-                bars->mref[t] = m_new;                      // (this thread read the old value above: one array serves both directions)
-                m_other = m_prev;
+        // Two ways of sharing a tile between the CTA's two softmax warpgroups (thread = query row = TMEM lane in both):
+        // bf16: every tile is taken by both warpgroups, 64 keys each, so that a row has two threads; the halves' maxima are
+        // exchanged through shared memory every tile.  The work per key is higher (P and its rounding remainder), and this
+        // form measured 9 % faster (mixed 13B-shaped batch, tile kernel 0.556 -> 0.506 ms).
+        // fp16: the warpgroups take alternate tiles, a whole row per thread; the exponentials of one overlap the waits of the
+        // other.  Measured 8 % faster than the split form for fp16 (8 chunks of 512 rows, 40 heads: 930 vs 858 TFLOP/s).
+        if constexpr (BF16) {
+            const int w = (warp - 2) >> 2;                      // warpgroup: takes keys [64 w, 64 w + 64) of every tile
+            const int quarter = warp & 3;                       // TMEM lanes this warp may touch
+            const int t = quarter * 32 + lane;                  // query row inside this CTA's tile = TMEM lane
+            const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
+            const uint32_t tm_o = tmem + kColO + lane_sel;
+            const int wg_tid = (int)threadIdx.x - 64 - w * 128;
+            const float sc = a.scale_log2;
+            const bool wide_stores = ((reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.part_out)) & 31) == 0;
+            const uint32_t lead_o_free = lead(&bars->o_free), lead_p_ready = lead(&bars->p_ready[0]);
+            int g0 = 0;                                         // global index of the unit's first tile
+            int px = 0;                                         // meetings of this warp with its partner so far
+            bool ok = true;
+            // The two threads of a row (same lane of the two warps that share a lane quarter) meet: what each wrote to shared
+            // memory before is visible to the other afterwards.  A bounded mbarrier wait like every other wait of the kernel.
+            auto pair_sync = [&]() -> bool {
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->m_ready[w][quarter]);
+                if (lane == 0) mbar_arrive(&bars->pair_bar[quarter]);
+                const bool met = __all_sync(0xffffffffu, mbar_wait(&bars->pair_bar[quarter], px & 1, cx));
+                ++px;
+                return met;
+            };
+            PH_DECL(16);
+            PH_T0(tw0);
+            for (int un = 0; ok; ++un) {
+                const int unit = read_unit(un, true);
+                PH_ADD(0, tw0);
+                if (unit == -2) { ok = false; break; }
+                if (unit < 0) break;
+                const Unit u = decode_unit(a, items, unit);
+                const int i_row = u.row0 + (int)rank * kRows + t;   // row inside the chunk
+                const int last_key = min(u.P + i_row, u.kv_end - 1);
+                float m_ref = -INFINITY;                         // the row's reference maximum (both threads of the row hold the same value)
+                float l = 0.f;                                   // row sum over this thread's keys, in units of m_ref
+                for (int j = 0; j < u.n; ++j) {
+                    const int g = g0 + j, b = g % kSBuf;
+                    const int kb = u.kv_begin + j * kKeys + w * 64;                  // first key of this thread's half
+                    const uint32_t tm_s = tmem + b * 128 + lane_sel;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[b], (g / kSBuf) & 1, cx));
+                    if (!ok) break;
+                    PH_ADD(1, tw0);
+                    tc_fence_after();
+                    float s[64];
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) tmem_ld32(tm_s + w * 64 + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
+                    tmem_ld_wait();
 
-                const float neg_ref = (m_new == -INFINITY) ? 0.f : -m_new;
-                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                    // raw maximum (the scale is positive, so it commutes with max); four independent chains
+                    const int lim = last_key - kb;              // keys 0..lim of this half are visible to this row
+                    if (lim < 63) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t p[16];
-                    uint32_t pl[16];
+                        for (int k = 0; k < 64; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
+                    }
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int k = 0; k < 32; k += 2) {
-                        const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
-                        const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
-                        sum4[(k >> 1) & 3] += e0 + e1;
-                        p[k / 2] = pack2<BF16>(e0, e1);
-                        if constexpr (BF16) {
-                            const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
-                            const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
-                            pl[k / 2] = pack2<BF16>(r0, r1);
+                    for (int k = 0; k < 64; k += 8) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], fmaxf(s[k + 2 * v], s[k + 2 * v + 1]));
+                    }
+                    const float mx_half = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    PH_ADD(2, tw0);
+                    // the other half's maximum.  After this meeting both threads also have their scores in registers, so P
+                    // (which overwrites the score columns of BOTH halves) may be written
+                    bars->mx_x[g & 1][w][t] = mx_half;
+                    ok = pair_sync();
+                    if (!ok) break;
+                    const float mx = fmaxf(mx_half, bars->mx_x[g & 1][w ^ 1][t]) * sc;
+                    PH_ADD(3, tw0);
+                    // the reference moves only when this tile's maximum exceeds it by more than the threshold (same decision in
+                    // both threads of the row: same inputs)
+                    const float m_new = (mx > m_ref + kRescaleThreshold) ? mx : m_ref;
+                    const bool rescale = (m_new != m_ref) && (m_ref != -INFINITY);
+                    const float alpha = rescale ? fast_exp2(m_ref - m_new) : 1.f;
+                    if (m_ref != m_new) l *= (m_ref == -INFINITY) ? 0.f : alpha;
+                    m_ref = m_new;
+
+                    const float neg_ref = (m_new == -INFINITY) ? 0.f : -m_new;
+                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t p[16];
+                        uint32_t pl[16];
+#pragma unroll
+                        for (int k = 0; k < 32; k += 2) {
+                            const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
+                            const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
+                            sum4[(k >> 1) & 3] += e0 + e1;
+                            p[k / 2] = pack2<BF16>(e0, e1);
+                            if constexpr (BF16) {
+                                const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
+                                const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
+                                pl[k / 2] = pack2<BF16>(r0, r1);
+                            }
+                        }
+                        // keys 64 w + 32 c .. + 31 are words 32 w + 16 c .. + 15 of P (and of its remainder, 64 columns on)
+                        tmem_st16(tm_s + w * 32 + c * 16, p);
+                        if constexpr (BF16) tmem_st16(tm_s + 64 + w * 32 + c * 16, pl);
+                    }
+                    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    PH_ADD(4, tw0);
+
+                    if (__any_sync(0xffffffffu, rescale)) {
+                        // O holds the tiles before this one in units of the old reference; the previous tile's P V must have
+                        // finished.  Each thread of the row rescales its half of the columns
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(g - 1) % kSBuf], ((g - 1) / kSBuf) & 1, cx));
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tm_o + w * 64 + c * 32, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                            tmem_st32(tm_o + w * 64 + c * 32, o);
                         }
                     }
-                    tmem_st16(tm_s + c * 16, p);
-                    if constexpr (BF16) tmem_st16(tm_s + 64 + c * 16, pl);
-                }
-                // this warpgroup's row sum, brought to the current reference first
-                if (m_mine != m_new) {
-                    l *= (m_mine == -INFINITY) ? 0.f : fast_exp2(m_mine - m_new);
-                    m_mine = m_new;
-                }
-                l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                PH_ADD(4, tw0);
-
-                if (__any_sync(0xffffffffu, rescale)) {
-                    // O holds the tiles before this one in units of m_prev; the previous tile's P V must have finished
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(g - 1) % kSBuf], ((g - 1) / kSBuf) & 1, cx));
+                    tmem_st_wait();
+                    PH_ADD(5, tw0);
+                    // this CTA's half of V tile g must have landed before the P V product may be issued (the MMA thread does
+                    // not look at the V ring itself)
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[g % kStagesV], (g / kStagesV) & 1, cx));
                     if (!ok) break;
-                    tc_fence_after();
-                    const float alpha = rescale ? fast_exp2(m_prev - m_new) : 1.f;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tm_o + c * 32, o);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                        tmem_st32(tm_o + c * 32, o);
+                    // a range that ends inside this tile: V rows past the range were not loaded (or hold stale slots); zero
+                    // them in this CTA's column half so that 0 * garbage cannot produce NaN
+                    if (u.kv_begin + (j + 1) * kKeys > u.kv_end) {
+                        unsigned char* vt = v_ring + (g % kStagesV) * kHalfBytes;
+                        const int first = u.kv_end - (u.kv_begin + j * kKeys);
+                        for (int idx = wg_tid + w * 128; idx < (kKeys - first) * 8; idx += 256) {
+                            const int row = first + idx / 8, part = idx % 8;       // 8 vectors of 16 bytes per 128-byte row
+                            *reinterpret_cast<uint4*>(vt + row * 128 + part * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                     }
+                    // one arrival per warp: every lane's P is in TMEM (wait::st) and fenced before the warp meets
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(lead_p_ready + b * 8);
+                    PH_ADD(6, tw0);
+#ifdef HAT_PHASE_TIMERS
+                    ph[15] += 1;
+#endif
                 }
-                tmem_st_wait();
-                PH_ADD(5, tw0);
-                // this CTA's half of V tile g must have landed before the P V product may be issued (the MMA thread does
-                // not look at the V ring itself)
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[g % kStagesV], (g / kStagesV) & 1, cx));
                 if (!ok) break;
-                // a range that ends inside this tile: V rows past the range were not loaded (or hold stale slots); zero
-                // them in this CTA's column half so that 0 * garbage cannot produce NaN
-                if (kb + kKeys > u.kv_end) {
-                    unsigned char* vt = v_ring + (g % kStagesV) * kHalfBytes;
-                    const int first = u.kv_end - kb;
-                    for (int idx = wg_tid; idx < (kKeys - first) * 8; idx += 128) {
-                        const int row = first + idx / 8, part = idx % 8;       // 8 vectors of 16 bytes per 128-byte row
-                        *reinterpret_cast<uint4*>(vt + row * 128 + part * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-                }
-                // one arrival per warp: every lane's P is in TMEM (wait::st) and fenced before the warp meets
+                // ---- end of the unit: the two threads of a row add their row sums (both in units of the same reference),
+                // and each stores its half of the columns
+                const int up = un & 1;
+                const int g_last = g0 + u.n - 1;
+                bars->lsum2[up][w][t] = l;
+                ok = pair_sync();
+                if (!ok) break;
+                const float l_tot = l + bars->lsum2[up][w ^ 1][t];
+                const float m_fin = m_ref;
+                PH_ADD(7, tw0);
+                // the last P V of the unit
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[g_last % kSBuf], (g_last / kSBuf) & 1, cx));
+                if (!ok) break;
+                PH_ADD(8, tw0);
+                tc_fence_after();
+                float o[64];                                    // this warpgroup's half of the columns
+#pragma unroll
+                for (int c = 0; c < 2; ++c) tmem_ld32(tm_o + w * 64 + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
+                tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_remote(lead_p_ready + b * 8);
-                PH_ADD(6, tw0);
-#ifdef HAT_PHASE_TIMERS
-                ph[15] += 1;
-#endif
-            }
-            if (!ok) break;
-            // ---- end of the unit.  The warpgroup that did not take the last tile hands its row sum over (it is in units
-            // of the reference the last tile read as m_prev); the other one adds its own, hands the total back and
-            // writes the lse.  Each then stores its half of the columns.
-            const int up = un & 1;
-            const int g_last = g0 + u.n - 1;
-            const bool took_last = (g_last & 1) == w;
-            float l_tot, m_fin = m_mine;
-            if (!took_last) {
-                bars->lsum[up][t] = l;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->fin_ready[w][quarter]);
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->fin_ready[w ^ 1][quarter], un & 1, cx));
-                if (!ok) break;
-                l_tot = bars->lsum[up][t];
-            } else {
-                ok = __all_sync(0xffffffffu, mbar_wait(&bars->fin_ready[w ^ 1][quarter], un & 1, cx));
-                if (!ok) break;
-                const float l_other = bars->lsum[up][t];
-                l_tot = l;
-                if (u.n > 1 && m_other != -INFINITY) l_tot += l_other * fast_exp2(m_other - m_fin);
-                bars->lsum[up][t] = l_tot;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->fin_ready[w][quarter]);
-            }
-            PH_ADD(7, tw0);
-            // the last P V of the unit
-            ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[g_last % kSBuf], (g_last / kSBuf) & 1, cx));
-            if (!ok) break;
-            PH_ADD(8, tw0);
-            tc_fence_after();
-            float o[64];                                    // this warpgroup's half of the columns
+                if (lane == 0) mbar_arrive_remote(lead_o_free);
+                if (i_row < u.C) {
+                    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+                    float* obase; float* lbase; int64_t orow;
+                    if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
+                    else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
+                    HAT_CHECK(orow >= 0 && orow < (u.part < 0 ? (int64_t)a.plan.total_rows : a.part_rows), cx.status);
+                    if (u.part < 0 && a.out16 != nullptr) {
+                        // final rows in the 16-bit output type: 128 bytes per row and warpgroup
+                        uint16_t* dst16 = static_cast<uint16_t*>(a.out16) + (orow * H + u.h) * kD + w * 64;
+                        const bool wide16 = (reinterpret_cast<uintptr_t>(a.out16) & 31) == 0;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) tmem_ld32(tm_o + w * 64 + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(lead_o_free);
-            if (i_row < u.C) {
-                const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-                float* obase; float* lbase; int64_t orow;
-                if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
-                else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
-                HAT_CHECK(orow >= 0 && orow < (u.part < 0 ? (int64_t)a.plan.total_rows : a.part_rows), cx.status);
-                if (u.part < 0 && a.out16 != nullptr) {
-                    // final rows in the 16-bit output type: 128 bytes per row and warpgroup
-                    uint16_t* dst16 = static_cast<uint16_t*>(a.out16) + (orow * H + u.h) * kD + w * 64;
-                    const bool wide16 = (reinterpret_cast<uintptr_t>(a.out16) & 31) == 0;
+                        for (int k = 0; k < 64; k += 16) {
+                            uint32_t wd[8];
 #pragma unroll
-                    for (int k = 0; k < 64; k += 16) {
-                        uint32_t wd[8];
+                            for (int e = 0; e < 8; ++e) wd[e] = pack_out16(o[k + 2 * e] * inv, o[k + 2 * e + 1] * inv, a.out16_bf16);
+                            if (wide16) {
+                                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
+                                             ::"l"(dst16 + k), "r"(wd[0]), "r"(wd[1]), "r"(wd[2]), "r"(wd[3]), "r"(wd[4]), "r"(wd[5]), "r"(wd[6]), "r"(wd[7]) : "memory");
+                            } else {
+                                *reinterpret_cast<uint4*>(dst16 + k) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                                *reinterpret_cast<uint4*>(dst16 + k + 8) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+                            }
+                        }
+                    } else {
+                        float* dst = obase + (orow * H + u.h) * kD + w * 64;
+                        if (wide_stores) {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) wd[e] = pack_out16(o[k + 2 * e] * inv, o[k + 2 * e + 1] * inv, a.out16_bf16);
-                        if (wide16) {
-                            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
-                                         ::"l"(dst16 + k), "r"(wd[0]), "r"(wd[1]), "r"(wd[2]), "r"(wd[3]), "r"(wd[4]), "r"(wd[5]), "r"(wd[6]), "r"(wd[7]) : "memory");
+                            for (int k = 0; k < 64; k += 8)
+                                st_global_v8(dst + k, o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv, o[k + 4] * inv,
+                                             o[k + 5] * inv, o[k + 6] * inv, o[k + 7] * inv);
                         } else {
-                            *reinterpret_cast<uint4*>(dst16 + k) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-                            *reinterpret_cast<uint4*>(dst16 + k + 8) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+#pragma unroll
+                            for (int k = 0; k < 64; k += 4)
+                                *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
                         }
                     }
-                } else {
-                    float* dst = obase + (orow * H + u.h) * kD + w * 64;
-                    if (wide_stores) {
-#pragma unroll
-                        for (int k = 0; k < 64; k += 8)
-                            st_global_v8(dst + k, o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv, o[k + 4] * inv,
-                                         o[k + 5] * inv, o[k + 6] * inv, o[k + 7] * inv);
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 64; k += 4)
-                            *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
-                    }
+                    if (w == 0) lbase[orow * H + u.h] = l_tot > 0.f ? (m_fin + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
                 }
-                if (took_last) lbase[orow * H + u.h] = l_tot > 0.f ? (m_fin + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
-            }
-            g0 += u.n;
-            PH_ADD(9, tw0);
+                g0 += u.n;
+                PH_ADD(9, tw0);
 #ifdef HAT_PHASE_TIMERS
-            ph[14] += 1;
+                ph[14] += 1;
+#endif
+            }
+#ifdef HAT_PHASE_TIMERS
+            if (lane == 0 && quarter == 0) PH_FLUSH(16 + 16 * w, 16);
+#endif
+        } else {
+            const int w = (warp - 2) >> 2;                      // warpgroup: takes the tiles with g % 2 == w
+            const int quarter = warp & 3;                       // TMEM lanes this warp may touch
+            const int t = quarter * 32 + lane;                  // query row inside this CTA's tile = TMEM lane
+            const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
+            const uint32_t tm_o = tmem + kColO + lane_sel;
+            const int wg_tid = (int)threadIdx.x - 64 - w * 128;
+            const float sc = a.scale_log2;
+            const bool wide_stores = ((reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.part_out)) & 31) == 0;
+            const uint32_t lead_o_free = lead(&bars->o_free), lead_p_ready = lead(&bars->p_ready[0]);
+            int g0 = 0;                                         // global index of the unit's first tile
+            bool ok = true;
+            PH_DECL(16);
+            PH_T0(tw0);
+            for (int un = 0; ok; ++un) {
+                const int unit = read_unit(un, true);
+                PH_ADD(0, tw0);
+                if (unit == -2) { ok = false; break; }
+                if (unit < 0) break;
+                const Unit u = decode_unit(a, items, unit);
+                const int i_row = u.row0 + (int)rank * kRows + t;   // row inside the chunk
+                const int last_key = min(u.P + i_row, u.kv_end - 1);
+                float m_mine = -INFINITY, l = 0.f;               // reference this warpgroup's row sum is expressed in; the sum
+                float m_other = -INFINITY;                       // reference the other warpgroup's latest tile of this unit left
+                for (int j = (g0 & 1) == w ? 0 : 1; j < u.n; j += 2) {
+                    const int g = g0 + j, b = g % kSBuf;
+                    const int kb = u.kv_begin + j * kKeys;
+                    const uint32_t tm_s = tmem + b * 128 + lane_sel;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[b], (g / kSBuf) & 1, cx));
+                    if (!ok) break;
+                    PH_ADD(1, tw0);
+                    tc_fence_after();
+                    float s[kKeys];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, reinterpret_cast<uint32_t*>(s) + c * 32);
+                    tmem_ld_wait();
+
+                    // raw maximum (the scale is positive, so it commutes with max); four independent chains
+                    const int lim = last_key - kb;              // keys 0..lim of this tile are visible to this row
+                    if (lim < kKeys - 1) {
+#pragma unroll
+                        for (int k = 0; k < kKeys; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
+                    }
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int k = 0; k < kKeys; k += 8) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], fmaxf(s[k + 2 * v], s[k + 2 * v + 1]));
+                    }
+                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
+                    PH_ADD(2, tw0);
+                    // the reference the previous tile (the other warpgroup's) left behind
+                    float m_prev = -INFINITY;
+                    if (j > 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bars->m_ready[w ^ 1][quarter], ((g - 1) >> 1) & 1, cx));
+                        if (!ok) break;
+                        m_prev = bars->mref[t];
+                    }
+                    PH_ADD(3, tw0);
+                    // move it only when this tile's maximum exceeds it by more than the threshold
+                    const float m_new = (mx > m_prev + kRescaleThreshold) ? mx : m_prev;
+                    const bool rescale = (m_new != m_prev) && (m_prev != -INFINITY);
+                    bars->mref[t] = m_new;                      // (this thread read the old value above: one array serves both directions)
+                    m_other = m_prev;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->m_ready[w][quarter]);
+
+                    const float neg_ref = (m_new == -INFINITY) ? 0.f : -m_new;
+                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t p[16];
+                        uint32_t pl[16];
+#pragma unroll
+                        for (int k = 0; k < 32; k += 2) {
+                            const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
+                            const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
+                            sum4[(k >> 1) & 3] += e0 + e1;
+                            p[k / 2] = pack2<BF16>(e0, e1);
+                            if constexpr (BF16) {
+                                const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
+                                const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
+                                pl[k / 2] = pack2<BF16>(r0, r1);
+                            }
+                        }
+                        tmem_st16(tm_s + c * 16, p);
+                        if constexpr (BF16) tmem_st16(tm_s + 64 + c * 16, pl);
+                    }
+                    // this warpgroup's row sum, brought to the current reference first
+                    if (m_mine != m_new) {
+                        l *= (m_mine == -INFINITY) ? 0.f : fast_exp2(m_mine - m_new);
+                        m_mine = m_new;
+                    }
+                    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    PH_ADD(4, tw0);
+
+                    if (__any_sync(0xffffffffu, rescale)) {
+                        // O holds the tiles before this one in units of m_prev; the previous tile's P V must have finished
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(g - 1) % kSBuf], ((g - 1) / kSBuf) & 1, cx));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const float alpha = rescale ? fast_exp2(m_prev - m_new) : 1.f;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tm_o + c * 32, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+                            tmem_st32(tm_o + c * 32, o);
+                        }
+                    }
+                    tmem_st_wait();
+                    PH_ADD(5, tw0);
+                    // this CTA's half of V tile g must have landed before the P V product may be issued (the MMA thread does
+                    // not look at the V ring itself)
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->v_full[g % kStagesV], (g / kStagesV) & 1, cx));
+                    if (!ok) break;
+                    // a range that ends inside this tile: V rows past the range were not loaded (or hold stale slots); zero
+                    // them in this CTA's column half so that 0 * garbage cannot produce NaN
+                    if (kb + kKeys > u.kv_end) {
+                        unsigned char* vt = v_ring + (g % kStagesV) * kHalfBytes;
+                        const int first = u.kv_end - kb;
+                        for (int idx = wg_tid; idx < (kKeys - first) * 8; idx += 128) {
+                            const int row = first + idx / 8, part = idx % 8;       // 8 vectors of 16 bytes per 128-byte row
+                            *reinterpret_cast<uint4*>(vt + row * 128 + part * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                    }
+                    // one arrival per warp: every lane's P is in TMEM (wait::st) and fenced before the warp meets
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(lead_p_ready + b * 8);
+                    PH_ADD(6, tw0);
+#ifdef HAT_PHASE_TIMERS
+                    ph[15] += 1;
+#endif
+                }
+                if (!ok) break;
+                // ---- end of the unit.  The warpgroup that did not take the last tile hands its row sum over (it is in units
+                // of the reference the last tile read as m_prev); the other one adds its own, hands the total back and
+                // writes the lse.  Each then stores its half of the columns.
+                const int up = un & 1;
+                const int g_last = g0 + u.n - 1;
+                const bool took_last = (g_last & 1) == w;
+                float l_tot, m_fin = m_mine;
+                if (!took_last) {
+                    bars->lsum[up][t] = l;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->fin_ready[w][quarter]);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->fin_ready[w ^ 1][quarter], un & 1, cx));
+                    if (!ok) break;
+                    l_tot = bars->lsum[up][t];
+                } else {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->fin_ready[w ^ 1][quarter], un & 1, cx));
+                    if (!ok) break;
+                    const float l_other = bars->lsum[up][t];
+                    l_tot = l;
+                    if (u.n > 1 && m_other != -INFINITY) l_tot += l_other * fast_exp2(m_other - m_fin);
+                    bars->lsum[up][t] = l_tot;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->fin_ready[w][quarter]);
+                }
+                PH_ADD(7, tw0);
+                // the last P V of the unit
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[g_last % kSBuf], (g_last / kSBuf) & 1, cx));
+                if (!ok) break;
+                PH_ADD(8, tw0);
+                tc_fence_after();
+                float o[64];                                    // this warpgroup's half of the columns
+#pragma unroll
+                for (int c = 0; c < 2; ++c) tmem_ld32(tm_o + w * 64 + c * 32, reinterpret_cast<uint32_t*>(o) + c * 32);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(lead_o_free);
+                if (i_row < u.C) {
+                    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+                    float* obase; float* lbase; int64_t orow;
+                    if (u.part < 0) { obase = a.out; lbase = a.lse; orow = u.row_base + i_row; }
+                    else { obase = a.part_out; lbase = a.part_lse; orow = u.part + (i_row - u.row0); }
+                    HAT_CHECK(orow >= 0 && orow < (u.part < 0 ? (int64_t)a.plan.total_rows : a.part_rows), cx.status);
+                    if (u.part < 0 && a.out16 != nullptr) {
+                        // final rows in the 16-bit output type: 128 bytes per row and warpgroup
+                        uint16_t* dst16 = static_cast<uint16_t*>(a.out16) + (orow * H + u.h) * kD + w * 64;
+                        const bool wide16 = (reinterpret_cast<uintptr_t>(a.out16) & 31) == 0;
+#pragma unroll
+                        for (int k = 0; k < 64; k += 16) {
+                            uint32_t wd[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) wd[e] = pack_out16(o[k + 2 * e] * inv, o[k + 2 * e + 1] * inv, a.out16_bf16);
+                            if (wide16) {
+                                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
+                                             ::"l"(dst16 + k), "r"(wd[0]), "r"(wd[1]), "r"(wd[2]), "r"(wd[3]), "r"(wd[4]), "r"(wd[5]), "r"(wd[6]), "r"(wd[7]) : "memory");
+                            } else {
+                                *reinterpret_cast<uint4*>(dst16 + k) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                                *reinterpret_cast<uint4*>(dst16 + k + 8) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+                            }
+                        }
+                    } else {
+                        float* dst = obase + (orow * H + u.h) * kD + w * 64;
+                        if (wide_stores) {
+#pragma unroll
+                            for (int k = 0; k < 64; k += 8)
+                                st_global_v8(dst + k, o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv, o[k + 4] * inv,
+                                             o[k + 5] * inv, o[k + 6] * inv, o[k + 7] * inv);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 64; k += 4)
+                                *reinterpret_cast<float4*>(dst + k) = make_float4(o[k] * inv, o[k + 1] * inv, o[k + 2] * inv, o[k + 3] * inv);
+                        }
+                    }
+                    if (took_last) lbase[orow * H + u.h] = l_tot > 0.f ? (m_fin + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
+                }
+                g0 += u.n;
+                PH_ADD(9, tw0);
+#ifdef HAT_PHASE_TIMERS
+                ph[14] += 1;
+#endif
+            }
+#ifdef HAT_PHASE_TIMERS
+            if (lane == 0 && quarter == 0) PH_FLUSH(16 + 16 * w, 16);
 #endif
         }
-#ifdef HAT_PHASE_TIMERS
-        if (lane == 0 && quarter == 0) PH_FLUSH(16 + 16 * w, 16);
-#endif
     }
 
     // both CTAs are done with each other's barriers, and every MMA has finished, before tensor memory is freed
