@@ -631,26 +631,34 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
                     m_ref = m_new;
 
                     const float neg_ref = (m_new == -INFINITY) ? 0.f : -m_new;
-                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                    // packed fp32 arithmetic (two values per instruction) for the scale, the row sum and the remainder
+                    const uint64_t sc2 = f2_pack(sc, sc), neg2 = f2_pack(neg_ref, neg_ref);
+                    uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         uint32_t p[16];
                         uint32_t pl[16];
 #pragma unroll
                         for (int k = 0; k < 32; k += 2) {
-                            const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
-                            const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
-                            sum4[(k >> 1) & 3] += e0 + e1;
+                            float x0, x1;
+                            f2_unpack(f2_fma(f2_pack(s[c * 32 + k], s[c * 32 + k + 1]), sc2, neg2), x0, x1);
+                            const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
+                            const uint64_t e2 = f2_pack(e0, e1);
+                            sum2[(k >> 1) & 3] = f2_add(sum2[(k >> 1) & 3], e2);
                             p[k / 2] = pack2<BF16>(e0, e1);
-                            if constexpr (BF16) {
-                                const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
-                                const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
-                                pl[k / 2] = pack2<BF16>(r0, r1);
-                            }
+                            float r0, r1;
+                            f2_unpack(f2_sub(e2, f2_pack(__uint_as_float(p[k / 2] << 16), __uint_as_float(p[k / 2] & 0xffff0000u))), r0, r1);
+                            pl[k / 2] = pack2<BF16>(r0, r1);
                         }
                         // keys 64 w + 32 c .. + 31 are words 32 w + 16 c .. + 15 of P (and of its remainder, 64 columns on)
                         tmem_st16(tm_s + w * 32 + c * 16, p);
-                        if constexpr (BF16) tmem_st16(tm_s + 64 + w * 32 + c * 16, pl);
+                        tmem_st16(tm_s + 64 + w * 32 + c * 16, pl);
+                    }
+                    float sum4[4];
+                    {
+                        float a0, a1, b0, b1, c0, c1, d0, d1;
+                        f2_unpack(sum2[0], a0, a1); f2_unpack(sum2[1], b0, b1); f2_unpack(sum2[2], c0, c1); f2_unpack(sum2[3], d0, d1);
+                        sum4[0] = a0 + a1; sum4[1] = b0 + b1; sum4[2] = c0 + c1; sum4[3] = d0 + d1;
                     }
                     l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                     PH_ADD(4, tw0);
