@@ -645,10 +645,10 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
                             const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
                             const uint64_t e2 = f2_pack(e0, e1);
                             sum2[(k >> 1) & 3] = f2_add(sum2[(k >> 1) & 3], e2);
-                            p[k / 2] = pack2<BF16>(e0, e1);
+                            p[k / 2] = pack2<true>(e0, e1);
                             float r0, r1;
                             f2_unpack(f2_sub(e2, f2_pack(__uint_as_float(p[k / 2] << 16), __uint_as_float(p[k / 2] & 0xffff0000u))), r0, r1);
-                            pl[k / 2] = pack2<BF16>(r0, r1);
+                            pl[k / 2] = pack2<true>(r0, r1);
                         }
                         // keys 64 w + 32 c .. + 31 are words 32 w + 16 c .. + 15 of P (and of its remainder, 64 columns on)
                         tmem_st16(tm_s + w * 32 + c * 16, p);
@@ -847,21 +847,14 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t p[16];
-                        uint32_t pl[16];
 #pragma unroll
                         for (int k = 0; k < 32; k += 2) {
                             const float e0 = fast_exp2(fmaf(s[c * 32 + k], sc, neg_ref));
                             const float e1 = fast_exp2(fmaf(s[c * 32 + k + 1], sc, neg_ref));
                             sum4[(k >> 1) & 3] += e0 + e1;
-                            p[k / 2] = pack2<BF16>(e0, e1);
-                            if constexpr (BF16) {
-                                const float r0 = e0 - __uint_as_float(p[k / 2] << 16);
-                                const float r1 = e1 - __uint_as_float(p[k / 2] & 0xffff0000u);
-                                pl[k / 2] = pack2<BF16>(r0, r1);
-                            }
+                            p[k / 2] = pack2<false>(e0, e1);
                         }
                         tmem_st16(tm_s + c * 16, p);
-                        if constexpr (BF16) tmem_st16(tm_s + 64 + c * 16, pl);
                     }
                     // this warpgroup's row sum, brought to the current reference first
                     if (m_mine != m_new) {
