@@ -525,7 +525,10 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
             if (C % 256 != 0 && C % 256 <= 128) all_wide = false;
             wide_tiles += (C + 255) / 256;
         }
-        if (all_wide && wide_tiles * p->num_heads >= 2 * (int64_t)num_sms) tile_kernel = 3;
+        // measured (chunks of 512 and 256 rows, 40 heads): for bf16 the pair kernel is the faster one at every batch size
+        // (1 to 8 chunks: 9 to 26 %), for fp16 from about 1.5 units per SM on (equal at 160 units, 2.5 % at 240, 16 % at 320)
+        const int64_t least = p->dtype == HAT_DTYPE_BF16 ? 1 : 3 * (int64_t)num_sms / 2;
+        if (all_wide && wide_tiles > 0 && wide_tiles * p->num_heads >= least) tile_kernel = 3;
     }
     if (const char* k = std::getenv("HAT_PREFILL_KERNEL")) {
         if (use_tc5 && p->head_dim == 128 && std::strcmp(k, "pair") == 0) tile_kernel = 3;

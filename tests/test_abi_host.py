@@ -242,20 +242,25 @@ def test_static_entry_point_clamps_unvalidated_lengths(hat_lib):
 
 
 def test_choice_of_the_tile_kernel(hat_lib):
-    """The CTA-pair kernel takes batches whose every unit fills both 128-row halves and that give the 74 pairs at least
-    two rounds of units; chunks of 64 or 128 rows, small batches and head_dim 64 keep the one-CTA tcgen05 kernel."""
-    def info(prefix, chunk, H, d=128):
+    """The CTA-pair kernel takes batches whose every unit fills both 128-row halves: for bf16 whatever their size, for
+    fp16 from 1.5 units per SM on; chunks of 64 or 128 rows and head_dim 64 keep the one-CTA tcgen05 kernel."""
+    def info(prefix, chunk, H, d=128, dtype="bf16"):
         rng = np.random.Generator(np.random.PCG64(3))
         table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=2)
-        c = B.make_cache_desc("bf16", num_pages, H, d, H * 16 * d, d, 16 * d)
+        c = B.make_cache_desc(dtype, num_pages, H, d, H * 16 * d, d, 16 * d)
         cu = np.concatenate([[0], np.cumsum(chunk)]).astype(np.int32)
         p = B.hat_plan_create(c, H, cu, np.asarray(prefix, np.int32), np.asarray(chunk, np.int32), table,
                               B.HAT_PLAN_HOST_ONLY)
         return B.hat_plan_get_info(p).as_dict()
-    assert info([100] * 8, [512] * 8, 40)["prefill_kernel"] == 3              # 16 wide units x 40 heads = 640 >= 296
+    assert info([100] * 8, [512] * 8, 40)["prefill_kernel"] == 3              # 16 wide units x 40 heads
     assert info([100] * 8 + [700] * 4, [512] * 8 + [4] * 4, 40)["prefill_kernel"] == 3   # short chunks do not matter
     assert info([100] * 8, [512] * 7 + [384], 40)["prefill_kernel"] == 1       # 384 = 256 + 128: a unit would idle half a pair
     assert info([100] * 8, [512] * 7 + [400], 40)["prefill_kernel"] == 3       # 400 = 256 + 144: both halves in use
     assert info([100] * 8, [128] * 8, 40)["prefill_kernel"] == 1
-    assert info([100] * 2, [512] * 2, 32)["prefill_kernel"] == 1               # 4 x 32 = 128 units < 296
+    assert info([100] * 2, [512] * 2, 32)["prefill_kernel"] == 3               # bf16: small batches too
+    assert info([100], [256], 8)["prefill_kernel"] == 3
+    assert info([100] * 2, [512] * 2, 32, dtype="fp16")["prefill_kernel"] == 1   # fp16: 4 x 32 = 128 units < 222
+    assert info([100] * 3, [512] * 3, 40, dtype="fp16")["prefill_kernel"] == 3   # 6 x 40 = 240
+    assert info([100] * 8, [512] * 8, 40, dtype="fp16")["prefill_kernel"] == 3
+    assert info([100] * 8, [4] * 8, 40)["prefill_kernel"] == 1                 # no tile-class chunk at all
     assert info([100] * 8, [512] * 8, 40, d=64)["prefill_kernel"] == 1
