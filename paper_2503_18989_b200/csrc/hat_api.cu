@@ -512,9 +512,9 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
                                        cache->stride_token, cache->stride_head);
     p->num_sms = num_sms;
     // Which tcgen05 tile kernel: the CTA-pair kernel (cta_group::2) shares every K/V tile between the two 128-row halves
-    // of a 256-row unit and is the faster one when every unit fills both halves and there are at least two rounds of
-    // units for the 74 pairs; batches with 64- or 128-row chunks (half of a pair would idle) and small batches keep the
-    // one-CTA kernel.  HAT_PREFILL_KERNEL = tc5 | pair | mma overrides.
+    // of a 256-row unit and is the faster one when every unit fills both halves (and, for fp16, the batch is not small);
+    // batches with 64- or 128-row chunks (half of a pair would idle) keep the one-CTA kernel.
+    // HAT_PREFILL_KERNEL = tc5 | pair | mma overrides.
     int tile_kernel = use_tc5 ? 1 : 0;
     if (use_tc5 && p->head_dim == 128) {
         bool all_wide = true;
