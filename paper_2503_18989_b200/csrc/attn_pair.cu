@@ -1017,13 +1017,14 @@ attn_pair_kernel(AttnArgs a, const WorkItem* __restrict__ items, int total_units
 
 }  // namespace
 
-cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream) {
+cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int num_units) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     const CUtensorMap *mk = nullptr, *mv = nullptr;
     const CUtensorMap* mq = plan_q_map(plan, args.q);
     if (!mq || !plan_pool_maps(plan, args.cache, &mk, &mv)) return cudaErrorInvalidValue;
     // the unit counter is zero at this point: the previous call's last CTA cleared it
-    const int total_units = (int)plan->tile_units.size();
+    const int total_units = num_units >= 0 ? num_units : (int)plan->tile_units.size();
+    if (total_units <= 0) return cudaSuccess;
     int32_t* counter = plan->dev.status + 1;
     // one cluster of two CTAs per pair of SMs, never more clusters than units
     int pairs = std::min(total_units, plan->num_sms / 2);

@@ -597,16 +597,18 @@ bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t
 }
 
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit,
-                            bool reset_counter) {
+                            bool reset_counter, int first_unit, int num_units, int counter_word) {
     const bool bf16 = plan->dtype == HAT_DTYPE_BF16;
     const CUtensorMap *mk = nullptr, *mv = nullptr;
     const CUtensorMap* mq = plan_q_map(plan, args.q);
     if (!mq || !plan_pool_maps(plan, args.cache, &mk, &mv)) return cudaErrorInvalidValue;
     // one CTA per SM draws units from a counter that is zero at this point: the previous call's last CTA cleared it
     // (reset_counter); a grid that joins another one on the same counter leaves it alone
-    const int total_units = (int)plan->tile_units.size();
-    int32_t* counter = plan->dev.status + 1;
+    const int total_units = num_units >= 0 ? num_units : (int)plan->tile_units.size() - first_unit;
+    if (total_units <= 0) return cudaSuccess;
+    int32_t* counter = plan->dev.status + counter_word;
     AttnArgs a2 = args;
+    a2.plan.tile_units = plan->dev.tile_units + first_unit;
     a2.tail_reset = reset_counter ? 1 : 0;
     int ctas = std::min(total_units, plan->num_sms);
     if (grid_limit > 0) ctas = std::min(ctas, grid_limit);

@@ -285,6 +285,7 @@ static void schedule(hat_plan* p, int num_sms, int tile_kernel) {
     // inside a request head by head, and for each head all items of the request one after the other, so that the row
     // blocks of one chunk (which read the same K/V of that head) run at the same time on neighbouring CTAs and meet in L2.
     p->tile_units.clear();
+    p->num_pair_units = 0;
     if (use_tc5) {
         std::vector<int> first_of_req(R, -1);
         std::vector<std::vector<int>> group;
@@ -293,9 +294,18 @@ static void schedule(hat_plan* p, int num_sms, int tile_kernel) {
             if (first_of_req[r] < 0) { first_of_req[r] = (int)group.size(); group.emplace_back(); }
             group[first_of_req[r]].push_back(i);
         }
-        for (const std::vector<int>& g : group)          // items are sorted longest first, so groups are too
-            for (int h = 0; h < H; ++h)
-                for (int i : g) p->tile_units.push_back((uint32_t)i | ((uint32_t)h << 16));
+        // With the CTA-pair kernel in use, units of more than 128 rows come first (they are its); units that would leave
+        // half of a pair idle follow and go to the one-CTA kernel.
+        auto rows_of = [&](int i) { return std::min(tile_rows, p->chunk_len[p->prefill_items[i].req] - p->prefill_items[i].row0); };
+        for (int pass = 0; pass < (tile_kernel == 3 ? 2 : 1); ++pass) {
+            for (const std::vector<int>& g : group)      // items are sorted longest first, so groups are too
+                for (int h = 0; h < H; ++h)
+                    for (int i : g) {
+                        if (tile_kernel == 3 && ((rows_of(i) > 128 || p->pair_takes_all) != (pass == 0))) continue;
+                        p->tile_units.push_back((uint32_t)i | ((uint32_t)h << 16));
+                    }
+            if (pass == 0) p->num_pair_units = tile_kernel == 3 ? (int)p->tile_units.size() : 0;
+        }
     }
 
     info.num_verify_items = (int32_t)p->verify_items.size();
@@ -327,7 +337,7 @@ static int upload(hat_plan* p) {
     size_t o_mr = blob_append(blob, p->merge_rows);
     size_t o_tu = blob_append(blob, p->tile_units);
     size_t o_tm = blob_append(blob, p->tree_mask);
-    std::vector<int32_t> status(4, 0);
+    std::vector<int32_t> status(8, 0);     // status word; (unit counter, finished CTAs) of the tile kernel; the same for a second tile grid; spare
     size_t o_st = blob_append(blob, status);
 
     cudaError_t e = cudaGetDevice(&p->device);
@@ -523,15 +533,19 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
             const int C = p->chunk_len[r];
             if (C <= 16) continue;
             if (C % 256 != 0 && C % 256 <= 128) all_wide = false;
-            wide_tiles += (C + 255) / 256;
+            wide_tiles += C / 256 + (C % 256 > 128 ? 1 : 0);
         }
         // measured (chunks of 512 and 256 rows, 40 heads): for bf16 the pair kernel is the faster one at every batch size
         // (1 to 8 chunks: 9 to 26 %), for fp16 from about 1.5 units per SM on (equal at 160 units, 2.5 % at 240, 16 % at 320)
-        const int64_t least = p->dtype == HAT_DTYPE_BF16 ? 1 : 3 * (int64_t)num_sms / 2;
-        if (all_wide && wide_tiles > 0 && wide_tiles * p->num_heads >= least) tile_kernel = 3;
+        // bf16: the units of more than 128 rows go to the pairs even when the batch also has narrower ones (those run on
+        // single CTAs behind them: a ragged bf16 batch measured 0.298 + 0.118 ms that way against 0.49 on either kernel alone)
+        const bool bf16 = p->dtype == HAT_DTYPE_BF16;
+        const int64_t least = bf16 ? 1 : 3 * (int64_t)num_sms / 2;
+        if ((all_wide || bf16) && wide_tiles > 0 && wide_tiles * p->num_heads >= least) tile_kernel = 3;
     }
+    p->pair_takes_all = false;
     if (const char* k = std::getenv("HAT_PREFILL_KERNEL")) {
-        if (use_tc5 && p->head_dim == 128 && std::strcmp(k, "pair") == 0) tile_kernel = 3;
+        if (use_tc5 && p->head_dim == 128 && std::strcmp(k, "pair") == 0) { tile_kernel = 3; p->pair_takes_all = true; }
         else if (use_tc5 && std::strcmp(k, "tc5") == 0) tile_kernel = 1;
     }
     schedule(p, num_sms, tile_kernel);
@@ -756,9 +770,15 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
         mark(1, 1);
     } else if (!plan->prefill_items.empty()) {
         mark(1, 0);
-        e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
-          : plan->info.prefill_kernel == 3 ? launch_attn_pair(plan, a, s)
-                                           : launch_attn_mma(plan, a, /*verify_class=*/false, s);
+        if (plan->info.prefill_kernel == 3) {
+            // units of more than 128 rows on CTA pairs, the others (if any) on single CTAs behind them
+            e = launch_attn_pair(plan, a, s, plan->num_pair_units);
+            if (e == cudaSuccess)
+                e = launch_attn_tc5(plan, a, s, 0, true, plan->num_pair_units, -1, /*counter_word=*/3);
+        } else {
+            e = plan->info.prefill_kernel == 1 ? launch_attn_tc5(plan, a, s)
+                                               : launch_attn_mma(plan, a, /*verify_class=*/false, s);
+        }
         if (e != cudaSuccess) return cuda_fail(e);
         mark(1, 1);
     }
@@ -894,7 +914,7 @@ int hat_last_device_status(const hat_plan* plan, void* stream, int* out) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int32_t word = 0;
     cudaError_t e = cudaMemcpyAsync(&word, plan->dev.status, sizeof word, cudaMemcpyDeviceToHost, s);
-    if (e == cudaSuccess) e = cudaMemsetAsync(plan->dev.status, 0, 4 * sizeof word, s);     // status, unit counter, finished CTAs
+    if (e == cudaSuccess) e = cudaMemsetAsync(plan->dev.status, 0, 8 * sizeof word, s);     // status, unit counters, finished CTAs
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
     *out = word == 0 ? HAT_OK : (word & 1) ? HAT_ERR_DEVICE_TIMEOUT : HAT_ERR_DEVICE_BOUNDS;

@@ -174,6 +174,8 @@ struct hat_plan {
     std::vector<int32_t> cu_chunk, prefix_len, chunk_len, block_table, row_req;
     std::vector<hat::WorkItem> verify_items, prefill_items;
     std::vector<uint32_t> tile_units;   // (item, head) of every unit of the tcgen05 tile kernels, in the order they are drawn
+    bool pair_takes_all;                // HAT_PREFILL_KERNEL=pair: every unit goes to the CTA-pair kernel, narrow ones too (tests)
+    int num_pair_units;                 // CTA-pair kernel in use: the first num_pair_units units are its (more than 128 rows each), the rest go to the one-CTA kernel
     std::vector<hat::MergeRow> merge_rows;
     int64_t part_rows;          // partial rows in the workspace
     hat_plan_info info;
@@ -216,10 +218,12 @@ cudaError_t launch_merge(const hat_plan* plan, const AttnArgs& args, int first_r
 bool tc5_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                           int64_t stride_head);
 // grid_limit > 0 caps the number of CTAs; reset_counter = false joins a grid that is already drawing units
+// first_unit / num_units (num_units < 0: all) select a part of the plan's unit list; counter_word: which pair of the
+// plan's status words (unit counter, finished CTAs) the grid uses
 cudaError_t launch_attn_tc5(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int grid_limit = 0,
-                            bool reset_counter = true);
+                            bool reset_counter = true, int first_unit = 0, int num_units = -1, int counter_word = 1);
 // tcgen05 tile kernel with 256-row units processed by clusters of two CTAs (cta_group::2), same layout requirements
-cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream);
+cudaError_t launch_attn_pair(const hat_plan* plan, const AttnArgs& args, cudaStream_t stream, int num_units = -1);   // the first num_units units
 // TMA-fed streaming kernel: whether a TMA descriptor can be built for this pool layout, and the launcher
 bool stream_layout_supported(int dtype, int head_dim, int num_pages, int H, int64_t stride_page, int64_t stride_token,
                              int64_t stride_head);

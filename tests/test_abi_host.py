@@ -242,8 +242,9 @@ def test_static_entry_point_clamps_unvalidated_lengths(hat_lib):
 
 
 def test_choice_of_the_tile_kernel(hat_lib):
-    """The CTA-pair kernel takes batches whose every unit fills both 128-row halves: for bf16 whatever their size, for
-    fp16 from 1.5 units per SM on; chunks of 64 or 128 rows and head_dim 64 keep the one-CTA tcgen05 kernel."""
+    """The CTA-pair kernel takes the units of more than 128 rows: for bf16 in every batch that has some (narrower units
+    of the same batch run on single CTAs), for fp16 only when every unit is that wide and there are at least 1.5 of
+    them per SM; head_dim 64 keeps the one-CTA tcgen05 kernel."""
     def info(prefix, chunk, H, d=128, dtype="bf16"):
         rng = np.random.Generator(np.random.PCG64(3))
         table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=2)
@@ -254,9 +255,10 @@ def test_choice_of_the_tile_kernel(hat_lib):
         return B.hat_plan_get_info(p).as_dict()
     assert info([100] * 8, [512] * 8, 40)["prefill_kernel"] == 3              # 16 wide units x 40 heads
     assert info([100] * 8 + [700] * 4, [512] * 8 + [4] * 4, 40)["prefill_kernel"] == 3   # short chunks do not matter
-    assert info([100] * 8, [512] * 7 + [384], 40)["prefill_kernel"] == 1       # 384 = 256 + 128: a unit would idle half a pair
+    assert info([100] * 8, [512] * 7 + [384], 40)["prefill_kernel"] == 3       # bf16: the 128-row unit of the 384 goes to a single CTA
     assert info([100] * 8, [512] * 7 + [400], 40)["prefill_kernel"] == 3       # 400 = 256 + 144: both halves in use
-    assert info([100] * 8, [128] * 8, 40)["prefill_kernel"] == 1
+    assert info([100] * 8, [128] * 8, 40)["prefill_kernel"] == 1               # nothing for a pair
+    assert info([100] * 8, [512] * 7 + [384], 40, dtype="fp16")["prefill_kernel"] == 1   # fp16: only batches of full units
     assert info([100] * 2, [512] * 2, 32)["prefill_kernel"] == 3               # bf16: small batches too
     assert info([100], [256], 8)["prefill_kernel"] == 3
     assert info([100] * 2, [512] * 2, 32, dtype="fp16")["prefill_kernel"] == 1   # fp16: 4 x 32 = 128 units < 222

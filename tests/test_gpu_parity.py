@@ -553,6 +553,30 @@ def test_calls_on_one_plan_from_two_streams_are_kept_in_order(cuda_device):
     ds.close()
 
 
+def test_a_bf16_batch_with_wide_and_narrow_units_uses_both_tile_kernels(cuda_device):
+    """bf16, head_dim 128: units of more than 128 rows run on CTA pairs and the narrower units of the same batch (a
+    128-row remainder of a 384-row chunk, chunks of 128 / 64 / 17 rows) on single CTAs in a second grid with its own
+    unit counter; every element against the oracle, twice in a row (the counters must be back at zero), also with key
+    ranges cut and merged."""
+    from paper_2503_18989_b200 import binding as B, runner
+    prefix = [0, 300, 1000, 37, 2000, 640, 90, 5000]
+    chunk = [512, 384, 128, 64, 300, 17, 4, 256]
+    sc = _manual("bf16", 2, 128, prefix, chunk, 71)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    assert ds.info["prefill_kernel"] == 3
+    kp, vp, want = oracle_replay(sc)
+    for _ in range(2):
+        ds.out.fill_(float("nan")); ds.lse.fill_(float("nan"))
+        ds.attend(fused_append=True)
+        go, gl = ds.results()
+        assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+        assert_parity(go, want[0][0], "wide + narrow out")
+        assert_parity(gl, want[0][1], "wide + narrow lse")
+    assert ds.canaries_intact()
+    ds.close()
+
+
 # ----------------------------------------------------------------------------
 # both tcgen05 tile kernels, whichever the plan would pick
 # ----------------------------------------------------------------------------
