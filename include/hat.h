@@ -128,7 +128,8 @@ typedef struct hat_plan_info {
     int32_t verify_split_len;    /* tokens per key range, streaming kernel */
     int32_t prefill_split_len;   /* tokens per key range, tile kernel (0 = unsplit) */
     int32_t prefill_tile_rows;   /* query rows per CTA of the tile kernel */
-    int32_t prefill_kernel;      /* 0 = mma.sync tile kernel, 1 = tcgen05 tile kernel (one CTA per unit), 3 = tcgen05 tile kernel by CTA pairs */
+    int32_t prefill_kernel;      /* 0 = mma.sync tile kernel, 1 = tcgen05 tile kernel (one CTA per unit), 3 = tcgen05 tile kernel by CTA pairs
+                                    for the units of more than 128 rows (narrower units of the same batch: one CTA per unit) */
     int64_t workspace_bytes;
     int64_t attn_flops;          /* 4*d*H_q*sum_r [C_r*P_r + C_r*(C_r+1)/2] (causal count, also when a tree mask is given) */
     int64_t kv_read_bytes;       /* 2*sum_r (P_r+C_r)*H_kv*d*elem: every visible K and V row read once per K/V head */
