@@ -492,10 +492,12 @@ def test_mixed_batch_with_the_tile_kernel_on_a_side_stream(cuda_device, monkeypa
     kernel runs, and a second tile grid joins on the freed SMs; same results, also when called back to back."""
     from paper_2503_18989_b200 import runner
     monkeypatch.setenv("HAT_SIDE_SMS", "56")
+    monkeypatch.setenv("HAT_PREFILL_KERNEL", "tc5")           # the mode exists for the one-CTA tile kernel
     sc = W.mixed_13b(num_prefill=5, prefill_chunk=384, max_prefill_prefix=3000, num_verify=12, min_verify_prefix=100,
                      max_verify_prefix=2000, H=4, seed=81)
     cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
     ds = runner.DeviceStep(cache, sc.steps[0])
+    assert ds.info["prefill_kernel"] == 1
     for _ in range(3):
         ds.attend()
     go, gl = ds.results()
