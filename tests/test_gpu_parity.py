@@ -579,6 +579,39 @@ def test_a_bf16_batch_with_wide_and_narrow_units_uses_both_tile_kernels(cuda_dev
     ds.close()
 
 
+@pytest.mark.parametrize("seed,group,out16", [(1, 1, False), (2, 2, False), (3, 1, True)])
+def test_random_bf16_batches_through_whatever_kernels_the_plan_picks(cuda_device, seed, group, out16):
+    """Random bf16 batches (chunks of 1 .. 700 rows, prefixes of 0 .. 3000 tokens, some not page multiples; grouped query
+    heads; 16-bit output): whichever mix of CTA-pair, one-CTA and streaming kernels and key-range cuts the plan picks,
+    every element against the oracle."""
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    rs = np.random.default_rng(100 + seed)
+    R = 9
+    chunk = [int(c) for c in rs.choice([1, 4, 16, 17, 64, 100, 128, 129, 200, 256, 300, 384, 512, 700], R)]
+    prefix = [int(rs.integers(0, 3001)) for _ in range(R)]
+    sc = _manual("bf16", 2, 128, prefix, chunk, 300 + seed, q_group=group)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    kp, vp, want = oracle_replay(sc)
+    if out16:
+        ds.attend16(fused_append=True)
+        torch.cuda.synchronize()
+        got = W.bits_to_f64(ds.out16.cpu().numpy().view(np.uint16), "bf16").reshape(want[0][0].shape)
+        err = np.abs(got - want[0][0])
+        assert np.all(err <= 2e-3 + np.abs(want[0][0]) * 2.0 ** -8), float(err.max())
+    else:
+        ds.attend(fused_append=True)
+        go, gl = ds.results()
+        assert_parity(go, want[0][0], f"random batch {seed} out")
+        assert_parity(gl, want[0][1], f"random batch {seed} lse")
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    assert ds.canaries_intact()
+    gk, gv = cache.pools_to_host()
+    assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+    ds.close()
+
+
 # ----------------------------------------------------------------------------
 # both tcgen05 tile kernels, whichever the plan would pick
 # ----------------------------------------------------------------------------
