@@ -528,20 +528,23 @@ int hat_plan_create(const hat_cache_desc* cache, const hat_batch_desc* batch, ha
     int tile_kernel = use_tc5 ? 1 : 0;
     if (use_tc5 && p->head_dim == 128) {
         bool all_wide = true;
-        int64_t wide_tiles = 0;
+        int64_t wide_tiles = 0, wide_keys = 0;
         for (int r = 0; r < R; ++r) {
             const int C = p->chunk_len[r];
             if (C <= 16) continue;
             if (C % 256 != 0 && C % 256 <= 128) all_wide = false;
-            wide_tiles += C / 256 + (C % 256 > 128 ? 1 : 0);
+            for (int row0 = 0; row0 < C; row0 += 256)
+                if (C - row0 > 128) { ++wide_tiles; wide_keys += p->prefix_len[r] + std::min(C, row0 + 256); }
         }
         // measured (chunks of 512 and 256 rows, 40 heads): for bf16 the pair kernel is the faster one at every batch size
         // (1 to 8 chunks: 9 to 26 %), for fp16 from about 1.5 units per SM on (equal at 160 units, 2.5 % at 240, 16 % at 320)
         // bf16: the units of more than 128 rows go to the pairs even when the batch also has narrower ones (those run on
         // single CTAs behind them: a ragged bf16 batch measured 0.298 + 0.118 ms that way against 0.49 on either kernel alone)
+        // fp16: pairs pay off only for long units (prefix 4000: +16 %; 8 chunks of 512 at prefix 2000: +4.5 %, at 1000: -2 %; a ragged batch's wide units, ~2300 keys on average with many short ones: -3 %)
         const bool bf16 = p->dtype == HAT_DTYPE_BF16;
         const int64_t least = bf16 ? 1 : 3 * (int64_t)num_sms / 2;
-        if ((all_wide || bf16) && wide_tiles > 0 && wide_tiles * p->num_heads >= least) tile_kernel = 3;
+        const bool long_units = bf16 || (wide_tiles > 0 && wide_keys / wide_tiles >= 2500);
+        if ((all_wide || bf16) && long_units && wide_tiles > 0 && wide_tiles * p->num_heads >= least) tile_kernel = 3;
     }
     p->pair_takes_all = false;
     if (const char* k = std::getenv("HAT_PREFILL_KERNEL")) {

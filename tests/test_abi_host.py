@@ -243,8 +243,8 @@ def test_static_entry_point_clamps_unvalidated_lengths(hat_lib):
 
 def test_choice_of_the_tile_kernel(hat_lib):
     """The CTA-pair kernel takes the units of more than 128 rows: for bf16 in every batch that has some (narrower units
-    of the same batch run on single CTAs), for fp16 only when every unit is that wide and there are at least 1.5 of
-    them per SM; head_dim 64 keeps the one-CTA tcgen05 kernel."""
+    of the same batch run on single CTAs), for fp16 only when every unit is that wide and long (2500 keys on average)
+    and there are at least 1.5 of them per SM; head_dim 64 keeps the one-CTA tcgen05 kernel."""
     def info(prefix, chunk, H, d=128, dtype="bf16"):
         rng = np.random.Generator(np.random.PCG64(3))
         table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=2)
@@ -262,7 +262,8 @@ def test_choice_of_the_tile_kernel(hat_lib):
     assert info([100] * 2, [512] * 2, 32)["prefill_kernel"] == 3               # bf16: small batches too
     assert info([100], [256], 8)["prefill_kernel"] == 3
     assert info([100] * 2, [512] * 2, 32, dtype="fp16")["prefill_kernel"] == 1   # fp16: 4 x 32 = 128 units < 222
-    assert info([100] * 3, [512] * 3, 40, dtype="fp16")["prefill_kernel"] == 3   # 6 x 40 = 240
-    assert info([100] * 8, [512] * 8, 40, dtype="fp16")["prefill_kernel"] == 3
+    assert info([4000] * 3, [512] * 3, 40, dtype="fp16")["prefill_kernel"] == 3   # 6 x 40 = 240 long units
+    assert info([4000] * 8, [512] * 8, 40, dtype="fp16")["prefill_kernel"] == 3
+    assert info([1000] * 8, [512] * 8, 40, dtype="fp16")["prefill_kernel"] == 1    # fp16 units of ~1400 keys: no gain on pairs
     assert info([100] * 8, [4] * 8, 40)["prefill_kernel"] == 1                 # no tile-class chunk at all
     assert info([100] * 8, [512] * 8, 40, d=64)["prefill_kernel"] == 1
