@@ -224,7 +224,10 @@ int hat_rope_q(const hat_plan* plan, const void* q, void* q_out, float theta, in
  *   q_out      device, [T][num_q_heads][head_dim], 16-byte aligned
  * head_dim 64 or 128.  Nothing is owned or kept by the library.  Errors:
  * INVALID_ARG, UNSUPPORTED (hidden not a multiple of 64, other head_dim), CUDA;
- * a device-side wait that ran out shows in hat_last_device_status.
+ * a device-side wait that ran out shows in hat_last_device_status.  The table of
+ * cosines and sines is kept with the plan and filled by the first call with a
+ * given theta (one more small kernel in that call); a call captured into a CUDA
+ * graph carries its own fill.  Like the attention calls, one call per plan at a time.
  */
 int hat_qkv_rope_append(const hat_cache_desc* cache, const hat_plan* plan, const void* x, int hidden, const void* w_qkv,
                         void* q_out, float theta, int interleaved, void* stream);

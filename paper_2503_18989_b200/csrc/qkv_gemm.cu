@@ -457,7 +457,20 @@ cudaError_t launch_qkv_gemm(const hat_plan* plan, const CacheView& cache, void* 
         // the table of cosines and sines depends on the plan's positions and on the base only: every layer of a step
         // uses the one its first call filled
         hat_plan* mp = const_cast<hat_plan*>(plan);
-        if (mp->rope_theta != theta) {
+        // Inside a stream capture nothing runs now: the fill becomes part of the captured graph (every replay refills the
+        // table, which is harmless) and the plan does not take the table as filled.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if ((e = cudaStreamIsCapturing(stream, &cap)) != cudaSuccess) return e;
+        const bool capturing = cap != cudaStreamCaptureStatusNone;
+        if (capturing) {
+            InvFreq fr;
+            for (int c = 0; c < 64; ++c) fr.f[c] = c < d / 2 ? std::pow((double)theta, -2.0 * c / d) : 0.0;
+            const int64_t total = (int64_t)T * (d / 2);
+            rope_table_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(plan->dev, d / 2, fr, mp->rope_table);
+            count_launch();
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            mp->rope_theta = 0.f;                // whoever calls next outside a capture fills it for itself
+        } else if (mp->rope_theta != theta) {
             InvFreq fr;
             for (int c = 0; c < 64; ++c) fr.f[c] = c < d / 2 ? std::pow((double)theta, -2.0 * c / d) : 0.0;
             const int64_t total = (int64_t)T * (d / 2);

@@ -324,3 +324,40 @@ def test_projection_kernel_gives_up_a_wait_and_the_context_stays_usable(cuda_dev
     want_q, _, _ = QO.qkv_rope(xb, wb, R.positions(st), dtype, hq, hkv, d)
     _assert_projected(q.cpu().numpy().view(np.uint16), want_q, dtype, "q rows after the self test", 0.97)
     ds.close()
+
+
+@pytest.mark.gpu
+def test_projection_call_captured_in_a_cuda_graph(cuda_device):
+    """The call neither allocates nor synchronises, so it can be captured; the captured graph carries its own fill of
+    the cosine / sine table, and a direct call afterwards (which finds the plan's table not yet filled) is correct too."""
+    import torch
+    from paper_2503_18989_b200 import binding as B, runner
+    dtype, d, hq, hkv, hidden = "bf16", 128, 2, 2, 192
+    prefix, chunk = [10, 777], [150, 40]
+    rng = np.random.Generator(np.random.PCG64(41))
+    table, num_pages = W._place_pages(rng, np.asarray(prefix) + np.asarray(chunk), slack_pages=2)
+    st = W._make_step(91, dtype, hkv, d, prefix, chunk, table, q_heads=hq)
+    sc = W._scenario("qkv", dtype, hkv, d, "paged", num_pages, [st], 91)
+    T = st.total_rows
+    xb, wb = W.projection_inputs(92, dtype, T, hidden, (hq + 2 * hkv) * d)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, st)
+    x_dev, w_dev = runner._dev_u16(xb, cuda_device), runner._dev_u16(wb, cuda_device)
+    q = torch.full((T, hq, d), -1, dtype=torch.int16, device=cuda_device)
+    side = torch.cuda.Stream(device=cuda_device)
+    side.wait_stream(torch.cuda.current_stream(cuda_device))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q, 10000.0, False, side.cuda_stream)
+    want_q, _, _ = QO.qkv_rope(xb, wb, R.positions(st), dtype, hq, hkv, d)
+    for _ in range(2):
+        q.fill_(-1)
+        graph.replay()
+        torch.cuda.synchronize()
+        _assert_projected(q.cpu().numpy().view(np.uint16), want_q, dtype, "q rows from the replayed graph", 0.97)
+    q.fill_(-1)
+    B.hat_qkv_rope_append(cache.desc, ds.plan, x_dev, hidden, w_dev, q, 10000.0, False)      # direct call after the capture
+    torch.cuda.synchronize()
+    _assert_projected(q.cpu().numpy().view(np.uint16), want_q, dtype, "q rows from a direct call", 0.97)
+    assert B.hat_last_device_status(ds.plan) == B.HAT_OK
+    ds.close()
