@@ -162,7 +162,11 @@ int64_t     hat_launch_count(void);
  * library keeps them ordered on the device: a call given another stream than
  * the plan's previous call first makes that stream wait for the previous call
  * (cudaStreamWaitEvent on an event the plan owns).  To overlap two steps on
- * one GPU, create two plans.
+ * one GPU, create two plans.  A call that is captured into a CUDA graph
+ * neither waits for nor records that event (a capture cannot depend on events
+ * of the world outside it): the caller orders the capturing stream behind the
+ * plan's earlier work before the capture begins, and replays of the graph
+ * behind each other as for any graph.
  * Errors: INVALID_ARG, UNSUPPORTED, OUT_OF_RANGE, CUDA, TOO_LARGE (more than 65535 work items of one class,
  * i.e. key ranges or 256-row tiles, in one batch).  *out is NULL on error.
  */

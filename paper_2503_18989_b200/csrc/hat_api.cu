@@ -702,13 +702,18 @@ static int run_attention(const hat_cache_desc* cache, const hat_plan* plan, cons
     cudaError_t e;
     // The plan's device state (unit counter, status word) serves one call at a time: a call on another stream than the
     // previous one is ordered behind it.
+    // A call that is being captured into a graph cannot wait for (or be waited for through) an event of the world outside
+    // the capture: there the caller orders the capturing stream behind the plan's earlier work before the capture begins.
     hat_plan* mplan = const_cast<hat_plan*>(plan);
-    if (plan->has_last && plan->last_stream != s && (e = cudaStreamWaitEvent(s, plan->ev_done, 0)) != cudaSuccess)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if ((e = cudaStreamIsCapturing(s, &cap)) != cudaSuccess) return cuda_fail(e);
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
+    if (!capturing && plan->has_last && plan->last_stream != s && (e = cudaStreamWaitEvent(s, plan->ev_done, 0)) != cudaSuccess)
         return cuda_fail(e);
     struct Done {
-        hat_plan* p; cudaStream_t s;
-        ~Done() { if (p->ev_done && cudaEventRecord(p->ev_done, s) == cudaSuccess) { p->last_stream = s; p->has_last = true; } }
-    } done{mplan, s};
+        hat_plan* p; cudaStream_t s; bool record;
+        ~Done() { if (record && p->ev_done && cudaEventRecord(p->ev_done, s) == cudaSuccess) { p->last_stream = s; p->has_last = true; } }
+    } done{mplan, s, !capturing};
     // optional event recorder: a start and an end event per slot (append, tile, streaming, merge)
     Timing* tm = plan->timing;
     int call = -1;

@@ -536,6 +536,34 @@ def test_the_call_can_be_captured_in_a_cuda_graph_and_replayed(cuda_device):
     assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
 
 
+def test_capture_on_another_stream_than_the_plans_earlier_calls(cuda_device):
+    """Warm-up calls on one stream, then the same plan's call captured on another stream (ordered behind the first by
+    the caller): the capture must not try to wait for the plan's own event of the warm-up calls."""
+    import torch
+    from paper_2503_18989_b200 import runner
+    sc = _manual("fp16", 2, 128, [100, 900, 40], [300, 4, 64], 93)
+    cache = runner.DeviceCache(sc.cache, sc.k_pool, sc.v_pool, cuda_device)
+    ds = runner.DeviceStep(cache, sc.steps[0])
+    cur = torch.cuda.current_stream(cuda_device)
+    for _ in range(2):
+        ds.attend(stream=cur.cuda_stream)                      # earlier calls: the plan remembers this stream
+    side = torch.cuda.Stream(device=cuda_device)
+    side.wait_stream(cur)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        ds.attend(stream=side.cuda_stream)
+    ds.out.fill_(float("nan")); ds.lse.fill_(float("nan"))
+    graph.replay()
+    go, gl = ds.results()
+    _, _, want = oracle_replay(sc)
+    assert_parity(go, want[0][0], "captured on another stream out")
+    assert_parity(gl, want[0][1], "captured on another stream lse")
+    ds.attend(stream=cur.cuda_stream)                          # and a plain call afterwards still works
+    go, gl = ds.results()
+    assert_parity(go, want[0][0], "plain call after the capture out")
+    ds.close()
+
+
 def test_calls_on_one_plan_from_two_streams_are_kept_in_order(cuda_device):
     """A plan serves one call at a time (its unit counter and status word are shared): calls handed different
     streams are ordered by the library itself, so alternating streams without any synchronisation is still correct."""
